@@ -1,0 +1,256 @@
+/*
+ * omnidraft.h — C ABI of the B200 (sm_100a) cross-vocabulary speculative
+ * verification step of OmniDraft (arXiv 2507.02659).
+ *
+ * One verification step, per sequence b of a batch (Algorithm 1, from the
+ * translation line to the free-token line):
+ *   1. od_map_proposals   translate the K_b proposed draft tokens into m_b
+ *                         target tokens t_i with draft probabilities q'(t_i)
+ *                         through the direct vocabulary map and the n-gram
+ *                         cache (Section 3.1, Eq. (1));
+ *   2. od_verify          temperature softmax of the m_b + 1 target-logit
+ *                         rows, acceptance ratio min(1, p(t_i)/q'(t_i)),
+ *                         accepted prefix length n_b (Algorithm 1);
+ *   3. od_sample_residual the extra token: drawn from norm(max(0, p - q'))
+ *                         with q'(.) of Eq. (2) at the first rejection, or
+ *                         from p (the free token) when everything was
+ *                         accepted.
+ *
+ * Conventions
+ *   - Every function returns an od_status (0 = OD_OK, negative = error). No
+ *     exceptions, no aborts, no output on stdout/stderr.
+ *   - "host" pointers are ordinary host memory read during the call.
+ *     "device" pointers are global memory of the context's GPU, owned by the
+ *     caller and neither retained nor freed by the library.
+ *   - The three step functions are asynchronous on `stream` (a cudaStream_t
+ *     passed as void*, NULL = the legacy default stream), allocate nothing and
+ *     never synchronise. Arguments are validated on the host (scalars,
+ *     alignment); data-dependent conditions are reported in device-side flag
+ *     words, never by a trap.
+ *   - A context holds scratch that its kernels share: calls on one context
+ *     must be ordered (one stream, or explicit dependencies). Use one context
+ *     per concurrent stream.
+ *   - Positions: arrays indexed [B, K_max] hold K_max entries per sequence,
+ *     of which the first K_b (inputs) or m_b (outputs) are meaningful.
+ *   - Random numbers: Philox4x32-10 (Salmon et al., SC'11) with key = the
+ *     sequence's 64-bit seed and counter = (step lo, step hi, position, tag);
+ *     u = (word0 >> 8) * 2^-24. tag 0 = acceptance test at `position`,
+ *     tag 1 = extra-token draw at `position`.
+ */
+#ifndef OMNIDRAFT_H
+#define OMNIDRAFT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct od_ctx od_ctx;
+
+enum od_status {
+    OD_OK = 0,
+    OD_ERR_INVALID_ARG = -1,       /* NULL pointer, size out of range */
+    OD_ERR_ALIGNMENT = -2,         /* logits base or stride not 16-byte aligned */
+    OD_ERR_MAP_NOT_INJECTIVE = -3, /* two draft ids map to one target id */
+    OD_ERR_BAD_CACHE_ENTRY = -4,   /* run length outside 2..4, id out of range */
+    OD_ERR_UNSUPPORTED = -5,       /* dtype, vocabulary too large for the cache key */
+    OD_ERR_CUDA = -6,              /* a CUDA runtime call failed */
+    OD_ERR_NOMEM = -7,
+    OD_ERR_STATE = -8              /* call out of order (e.g. no vocabulary map yet) */
+};
+
+enum od_dtype { OD_F32 = 0, OD_BF16 = 1 };
+
+/* tail_kind[b] written by od_map_proposals */
+enum od_tail {
+    OD_TAIL_COMPLETE = 0,      /* all K_b draft tokens were translated */
+    OD_TAIL_UNMAPPED_STOP = 1  /* translation stopped at a token with neither a
+                                  cache hit nor a direct map: position m_b is a
+                                  forced rejection */
+};
+
+/* counters[] accumulated (atomically added to) by od_map_proposals */
+enum od_counter {
+    OD_CNT_CACHE_HITS = 0,
+    OD_CNT_UNMAPPED_STOPS = 1,
+    OD_CNT_INVALID_IDS = 2,    /* draft ids outside [0, draft_vocab) */
+    OD_CNT_MAPPED_TOKENS = 3,  /* sum of m_b */
+    OD_CNT_COUNT = 4
+};
+
+/* verify_flags[b] written by od_verify */
+#define OD_VF_BOUNDARY_MASK 0x0000FFFFu /* bit i: |u_i - ratio_i| <= OD_TAU_ACCEPT */
+#define OD_VF_BAD_TEMPERATURE 0x00010000u
+#define OD_VF_NONFINITE 0x00020000u     /* a row sum is not finite and positive */
+
+/* sample_flags[b] written by od_sample_residual */
+#define OD_SF_BOUNDARY 0x1u        /* u*R within OD_TAU_SAMPLE*R of a CDF edge of the token */
+#define OD_SF_ZERO_MASS 0x2u       /* residual mass <= 0: drawn from p instead */
+#define OD_SF_BAD_TEMPERATURE 0x4u
+#define OD_SF_BONUS 0x10u          /* the token is the free token (n_b == m_b) */
+
+/* fp32 arithmetic can land on the other side of a decision than exact
+ * arithmetic only inside these margins; such decisions are flagged. */
+#define OD_TAU_ACCEPT 1.0e-5f
+#define OD_TAU_SAMPLE 2.0e-6
+
+#define OD_MAX_K 16      /* largest K_max */
+#define OD_NGRAM_MAX 4   /* longest cached run */
+
+/* ---- context ----------------------------------------------------------- */
+
+/* Create a context on CUDA device `device` for a draft vocabulary of
+ * `draft_vocab` ids and a target vocabulary of `target_vocab` ids, for
+ * batches of at most `max_batch` sequences with at most `max_k`
+ * (1..OD_MAX_K) proposed tokens each. Allocates the device-side scratch
+ * (tickets, partial row statistics, tile sums) once; synchronous. */
+int32_t od_create(od_ctx **ctx, int32_t device, int32_t draft_vocab,
+                  int32_t target_vocab, int32_t max_batch, int32_t max_k);
+
+/* Free everything the context owns. Synchronises the device first. */
+int32_t od_destroy(od_ctx *ctx);
+
+/* Direct vocabulary map t <-> d on the intersection of the vocabularies
+ * (Eq. (1), first case). host_map: int32[draft_vocab], target id or -1.
+ * Builds the inverse map, uploads both (synchronous). Rejects target ids
+ * outside [0, target_vocab) (INVALID_ARG) and maps that send two draft ids to
+ * one target id (MAP_NOT_INJECTIVE). */
+int32_t od_set_vocab_map(od_ctx *ctx, const int32_t *host_map);
+
+/* n-gram cache C = {(t, [d_1..d_n])} (Section 3.1). host_runs: int32[E,4],
+ * unused slots ignored; host_len: int32[E] in 2..4; host_target: int32[E].
+ * Builds an open-addressing table (32-slot groups, load <= 1/2) on the host,
+ * deterministically, and uploads it (synchronous). When a run appears twice
+ * the first entry wins (Algorithm 1 only inserts an unseen n-gram). E = 0
+ * installs an empty cache. Replaces any earlier cache. Needs
+ * draft_vocab <= 65535 when E > 0 (UNSUPPORTED otherwise): a run is packed
+ * into one 64-bit key, 16 bits per id. */
+int32_t od_cache_build(od_ctx *ctx, const int32_t *host_runs,
+                       const int32_t *host_len, const int32_t *host_target,
+                       int64_t E);
+
+/* Tuning knobs, mainly for experiments. Names: "verify_chunk_bytes" (bytes of
+ * one logit row given to one thread block, 0 = automatic), "sample_tiles_per_block"
+ * (0 = automatic). Unknown name: INVALID_ARG. */
+int32_t od_set_option(od_ctx *ctx, const char *name, int64_t value);
+
+/* ---- the step ----------------------------------------------------------- */
+
+/* Step 1 (Eq. (1); Algorithm 1, translation line). Scan d_0..d_{K_b-1} left to
+ * right; at each offset try the cached runs of length min(4, remaining)..2,
+ * longest first; on a hit emit (t, prod_j q(d_j)) and skip the run; otherwise
+ * emit the directly mapped token (map[d], q(d)); a token with neither ends the
+ * translation (OD_TAIL_UNMAPPED_STOP).
+ *   in  (device) draft_ids  int32[B,K_max]   proposed draft ids
+ *                draft_len  int32[B]         K_b, clamped to [0, K_max]
+ *                q_sel      float[B,K_max]   q(d_j) of each proposed token
+ *   out (device) tgt_ids    int32[B,K_max]   t_i, i < m_b
+ *                q_prime    float[B,K_max]   q'(t_i), i < m_b
+ *                span_start int32[B,K_max]   first draft position of piece i;
+ *                                            under UNMAPPED_STOP entry m_b is
+ *                                            the stopping position
+ *                span_len   int32[B,K_max]   draft tokens merged into piece i
+ *                m          int32[B]         number of translated tokens
+ *                tail_kind  uint8[B]         enum od_tail
+ *                counters   uint32[OD_CNT_COUNT], added to (may be NULL)
+ * Entries at positions >= m_b (beyond the stop entry) are left untouched. */
+int32_t od_map_proposals(od_ctx *ctx, int32_t B, int32_t K_max,
+                         const int32_t *draft_ids, const int32_t *draft_len,
+                         const float *q_sel, int32_t *tgt_ids, float *q_prime,
+                         int32_t *span_start, int32_t *span_len, int32_t *m,
+                         uint8_t *tail_kind, uint32_t *counters, void *stream);
+
+/* Step 2 (Algorithm 1, target-probability and rejection lines). For each
+ * sequence, rows 0..m_b of its logits are read exactly once:
+ * M_r = max_t x_t, S_r = sum_t exp((x_t - M_r)/T_b); for i < m_b
+ * p_sel_i = exp((x[t_i] - M_i)/T_b)/S_i, ratio_i = 1 if q'_i <= p_sel_i else
+ * p_sel_i/q'_i, accepted iff u_i < ratio_i; n_b = number of leading accepts.
+ *   in  (device) logits  fp32 or bf16, element (b, r, t) at
+ *                        b*seq_stride + r*row_stride + t (strides in elements);
+ *                        base and both strides must be multiples of 16 bytes;
+ *                        rows above m_b are never touched
+ *                tgt_ids, q_prime, span_len, m  as written by step 1
+ *                temperature float[B] (> 0, else BAD_TEMPERATURE is flagged
+ *                        and n_b = 0), seed uint64[B]
+ *   out (device) row_max, row_sum float[B,K_max+1]   rows 0..m_b
+ *                p_sel, ratio    float[B,K_max]      i < m_b
+ *                n_accepted, n_draft_accepted int32[B] (the latter = draft
+ *                        tokens covered by the accepted pieces)
+ *                verify_flags uint32[B] */
+int32_t od_verify(od_ctx *ctx, int32_t B, int32_t K_max, const void *logits,
+                  int32_t logit_dtype, int64_t row_stride, int64_t seq_stride,
+                  const int32_t *tgt_ids, const float *q_prime,
+                  const int32_t *span_len, const int32_t *m,
+                  const float *temperature, const uint64_t *seed, uint64_t step,
+                  float *row_max, float *row_sum, float *p_sel, float *ratio,
+                  int32_t *n_accepted, int32_t *n_draft_accepted,
+                  uint32_t *verify_flags, void *stream);
+
+/* Step 3 (notation paragraph of Section 3: residual; Eq. (2); Algorithm 1,
+ * rejection and free-token lines). Position j = n_b. If j < m_b, or j == m_b
+ * under UNMAPPED_STOP: r(t) = max(0, p_j(t) - q'_j(t)) where q'_j(.) is the
+ * drafter's row q_rows[b, span_start_j, .] carried through the inverse map (0
+ * outside the map's image), and, when piece j is a cached n-gram with token T
+ * and first sub-token d_1: q'_j(map[d_1]) = q(d_1) - q'(T) (if d_1 is mapped)
+ * and then q'_j(T) = q'(T). Otherwise (free token) r = p_m. The output is the
+ * smallest t whose inclusive cumulative sum exceeds u*R, R = sum_t r(t), in
+ * target-id order. If R <= 0 the token is drawn from p_j and ZERO_MASS is set.
+ *   in  (device) logits (as for od_verify), row_max, row_sum from step 2,
+ *                q_rows float[B,K_max,draft_vocab] drafter distributions,
+ *                draft_ids, tgt_ids, q_prime, span_start, span_len, m,
+ *                tail_kind from step 1, n_accepted from step 2,
+ *                temperature, seed, step as for step 2
+ *   out (device) out_token int32[B], resid_mass float[B] (R),
+ *                sample_flags uint32[B] */
+int32_t od_sample_residual(od_ctx *ctx, int32_t B, int32_t K_max,
+                           const void *logits, int32_t logit_dtype,
+                           int64_t row_stride, int64_t seq_stride,
+                           const float *row_max, const float *row_sum,
+                           const float *q_rows, const int32_t *draft_ids,
+                           const int32_t *tgt_ids, const float *q_prime,
+                           const int32_t *span_start, const int32_t *span_len,
+                           const int32_t *m, const uint8_t *tail_kind,
+                           const int32_t *n_accepted, const float *temperature,
+                           const uint64_t *seed, uint64_t step,
+                           int32_t *out_token, float *resid_mass,
+                           uint32_t *sample_flags, void *stream);
+
+/* ---- whole step from host memory ---------------------------------------- */
+
+/* Allocate device staging for od_step_host: inputs and outputs of one step of
+ * max_batch x max_k, logits of `logit_dtype` stored densely. Synchronous. */
+int32_t od_host_step_reserve(od_ctx *ctx, int32_t logit_dtype);
+
+/* Steps 1-3 on HOST buffers (pinned memory recommended): copies the inputs to
+ * the staging area, runs the three kernels, copies the results back, all on
+ * `stream`, and synchronises that stream before returning. Host layouts are
+ * the dense ones above (logits [B, K_max+1, target_vocab]). Outputs: host
+ * int32[B] each for n_accepted, n_draft_accepted, out_token; int32[B,K_max]
+ * tgt_ids; int32[B] m; uint32[B] verify_flags and sample_flags (any output may
+ * be NULL). Needs od_host_step_reserve with the same dtype. */
+int32_t od_step_host(od_ctx *ctx, int32_t B, int32_t K_max,
+                     const int32_t *draft_ids, const int32_t *draft_len,
+                     const float *q_sel, const float *q_rows,
+                     const void *logits, int32_t logit_dtype,
+                     const float *temperature, const uint64_t *seed,
+                     uint64_t step, int32_t *n_accepted,
+                     int32_t *n_draft_accepted, int32_t *out_token,
+                     int32_t *tgt_ids, int32_t *m, uint32_t *verify_flags,
+                     uint32_t *sample_flags, void *stream);
+
+/* ---- misc ---------------------------------------------------------------- */
+
+/* Number of thread blocks the last od_verify / od_sample_residual call on this
+ * context launched and the bytes of one row chunk (for benchmarks). which: 0 =
+ * verify grid size, 1 = verify chunk elements, 2 = sample grid size, 3 = sample
+ * tiles per block. */
+int64_t od_last_launch_info(const od_ctx *ctx, int32_t which);
+
+const char *od_status_string(int32_t status);
+int32_t od_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OMNIDRAFT_H */

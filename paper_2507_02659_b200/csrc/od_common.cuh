@@ -1,0 +1,160 @@
+// Shared declarations of the CUDA library: the context, device helpers
+// (Philox4x32-10, logit decoding, (max, sum) pair algebra) and the kernel
+// launchers implemented in od_map.cu / od_verify.cu / od_sample.cu.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "omnidraft.h"
+
+#define OD_WARP 32
+#define OD_GROUP 32                 // slots of one hash-table probe group
+#define OD_SAMPLE_TILE 2048         // elements of one residual-sampler tile
+#define OD_SAMPLE_THREADS 256
+#define OD_VERIFY_THREADS 256
+
+struct od_ctx {
+    int device;
+    int32_t v_q, v_p, max_batch, max_k;
+    int sm_count;
+
+    // vocabulary map (device)
+    int32_t *d_vocab_map;           // [v_q]
+    int32_t *d_inv_map;             // [v_p], -1 outside the image
+    bool have_map;
+
+    // n-gram cache: open addressing over groups of 32 slots
+    uint64_t *d_keys;               // [cap], 0 = empty
+    int32_t *d_vals;                // [cap]
+    int64_t cap;                    // power of two, multiple of 32, or 0
+
+    // od_verify scratch
+    float2 *d_partials;             // [max_batch*(max_k+1)*max_chunks] (max, sum)
+    unsigned int *d_row_ticket;     // [max_batch*(max_k+1)]
+    unsigned int *d_seq_ticket;     // [max_batch]
+    unsigned int *d_seq_bits;       // [max_batch][2]: accept bits | boundary bits << 16; misc
+    int32_t max_chunks;
+
+    // od_sample_residual scratch
+    double *d_tile_sums;            // [max_batch * tiles_per_row]
+    unsigned int *d_samp_ticket;    // [max_batch]
+    int32_t tiles_per_row;
+
+    // options
+    int64_t opt_verify_chunk_bytes;
+    int64_t opt_sample_tiles_per_block;
+
+    // last launch info
+    int64_t info[4];
+
+    // od_step_host staging (device)
+    bool host_reserved;
+    int32_t host_dtype;
+    void *s_logits;
+    float *s_q_rows, *s_q_sel, *s_temperature;
+    int32_t *s_draft_ids, *s_draft_len;
+    uint64_t *s_seed;
+    int32_t *s_tgt_ids, *s_span_start, *s_span_len, *s_m, *s_n_acc, *s_n_draft, *s_token;
+    float *s_q_prime, *s_row_max, *s_row_sum, *s_p_sel, *s_ratio, *s_mass;
+    uint8_t *s_tail;
+    uint32_t *s_vflags, *s_sflags;
+};
+
+// ---- launchers ------------------------------------------------------------
+cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids,
+                          const int32_t *draft_len, const float *q_sel, int32_t *tgt_ids,
+                          float *q_prime, int32_t *span_start, int32_t *span_len, int32_t *m,
+                          uint8_t *tail_kind, uint32_t *counters, cudaStream_t s);
+
+cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
+                             int32_t dtype, int64_t row_stride, int64_t seq_stride,
+                             const int32_t *tgt_ids, const float *q_prime,
+                             const int32_t *span_len, const int32_t *m,
+                             const float *temperature, const uint64_t *seed, uint64_t step,
+                             float *row_max, float *row_sum, float *p_sel, float *ratio,
+                             int32_t *n_accepted, int32_t *n_draft_accepted,
+                             uint32_t *flags, cudaStream_t s);
+
+cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
+                             int32_t dtype, int64_t row_stride, int64_t seq_stride,
+                             const float *row_max, const float *row_sum, const float *q_rows,
+                             const int32_t *draft_ids, const int32_t *tgt_ids,
+                             const float *q_prime, const int32_t *span_start,
+                             const int32_t *span_len, const int32_t *m,
+                             const uint8_t *tail_kind, const int32_t *n_accepted,
+                             const float *temperature, const uint64_t *seed, uint64_t step,
+                             int32_t *out_token, float *resid_mass, uint32_t *flags,
+                             cudaStream_t s);
+
+// 64-bit key of a run of draft ids: (id + 1) in 16 bits per position, first id
+// in the low bits. Never 0 for a non-empty run.
+__host__ __device__ inline uint64_t od_pack_run(const int32_t *ids, int len)
+{
+    uint64_t k = 0;
+    for (int j = 0; j < len; ++j) k |= (uint64_t)(uint32_t)(ids[j] + 1) << (16 * j);
+    return k;
+}
+
+// 64-bit finaliser of MurmurHash3 (Appleby, public domain): spreads the packed
+// key over the table's groups.
+__host__ __device__ inline uint64_t od_hash64(uint64_t h)
+{
+    h ^= h >> 33; h *= 0xff51afd7ed558ccdULL;
+    h ^= h >> 33; h *= 0xc4ceb9fe1a85ec53ULL;
+    h ^= h >> 33;
+    return h;
+}
+
+#ifdef __CUDACC__
+// ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) ----------------------
+__device__ __forceinline__ uint32_t od_philox_word0(uint32_t c0, uint32_t c1, uint32_t c2,
+                                                    uint32_t c3, uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        uint32_t n0 = hi1 ^ c1 ^ k0;
+        uint32_t n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+
+// uniform in [0,1) on the 24-bit grid for (seed, step, position, tag)
+__device__ __forceinline__ float od_uniform(uint64_t seed, uint64_t step, uint32_t position,
+                                            uint32_t tag)
+{
+    uint32_t w = od_philox_word0((uint32_t)step, (uint32_t)(step >> 32), position, tag,
+                                 (uint32_t)seed, (uint32_t)(seed >> 32));
+    return (float)(w >> 8) * (1.0f / 16777216.0f);
+}
+
+__device__ __forceinline__ float od_ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// (max, sum) of exp2((x - max) * scale): merge two partial pairs
+__device__ __forceinline__ void od_pair_merge(float &m, float &s, float m2, float s2, float scale)
+{
+    float nm = fmaxf(m, m2);
+    s = s * od_ex2((m - nm) * scale) + s2 * od_ex2((m2 - nm) * scale);
+    m = nm;
+}
+
+__device__ __forceinline__ float od_bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float od_bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+template <int DTYPE>
+__device__ __forceinline__ float od_load_logit(const void *row, int64_t t)
+{
+    if (DTYPE == OD_F32) return __ldg((const float *)row + t);
+    uint16_t h = __ldg((const unsigned short *)row + t);
+    return __uint_as_float((uint32_t)h << 16);
+}
+#endif  // __CUDACC__

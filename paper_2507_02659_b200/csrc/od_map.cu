@@ -1,0 +1,145 @@
+// Step 1: translation of the draft proposal into the target vocabulary
+// (Section 3.1, Eq. (1); Algorithm 1, translation line).
+//
+// One thread block per sequence, one warp per proposal offset. Warp s probes
+// the n-gram cache for the runs of length 4, 3, 2 that start at offset s: the
+// cache is an open-addressing table of 32-slot groups, a probe reads one group
+// with one coalesced 256-byte load (lane <-> slot) and resolves it with two
+// ballots (key match / empty slot). The first probes of the three lengths are
+// issued together so their latencies overlap. After a block barrier one thread
+// walks the proposal left to right, longest hit first, then the direct map,
+// and writes the mapped proposal. Integer work throughout, except the product
+// of at most four fp32 draft probabilities.
+#include "od_common.cuh"
+
+namespace {
+
+__device__ __forceinline__ int32_t probe_continue(const uint64_t *__restrict__ keys,
+                                                  const int32_t *__restrict__ vals,
+                                                  uint64_t ngroups, uint64_t key, uint64_t g,
+                                                  uint64_t k_lane, int lane)
+{
+    // resolves a lookup whose first group (already loaded into k_lane) is g;
+    // walks at most ngroups groups, so it ends on any table contents
+    for (uint64_t step = 0; step < ngroups; ++step) {
+        unsigned match = __ballot_sync(0xFFFFFFFFu, k_lane == key);
+        if (match) return __ldg(vals + g * OD_GROUP + (__ffs(match) - 1));
+        unsigned empty = __ballot_sync(0xFFFFFFFFu, k_lane == 0ULL);
+        if (empty) return -1;
+        g = (g + 1) & (ngroups - 1);
+        k_lane = __ldg(keys + g * OD_GROUP + lane);
+    }
+    return -1;
+}
+
+__global__ void __launch_bounds__(OD_MAX_K *OD_WARP)
+od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__ draft_ids,
+              const int32_t *__restrict__ draft_len, const float *__restrict__ q_sel,
+              const int32_t *__restrict__ vocab_map, const uint64_t *__restrict__ keys,
+              const int32_t *__restrict__ vals, int64_t cap, int32_t *__restrict__ tgt_ids,
+              float *__restrict__ q_prime, int32_t *__restrict__ span_start,
+              int32_t *__restrict__ span_len, int32_t *__restrict__ m_out,
+              uint8_t *__restrict__ tail_kind, uint32_t *__restrict__ counters)
+{
+    __shared__ int32_t s_ids[OD_MAX_K];
+    __shared__ int32_t s_hit[OD_MAX_K][OD_NGRAM_MAX + 1];   // [offset][length] -> target or -1
+
+    const int b = blockIdx.x;
+    if (b >= B) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int K = draft_len[b];
+    K = K < 0 ? 0 : (K > K_max ? K_max : K);
+
+    if (threadIdx.x < K_max) s_ids[threadIdx.x] = draft_ids[(size_t)b * K_max + threadIdx.x];
+    __syncthreads();
+
+    const int s = warp;
+    if (s < K) {
+        int32_t hit[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
+        if (cap > 0) {
+            const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
+            uint64_t key[OD_NGRAM_MAX + 1], grp[OD_NGRAM_MAX + 1], kl[OD_NGRAM_MAX + 1];
+            bool valid[OD_NGRAM_MAX + 1];
+            // ids of a run must lie in the draft vocabulary; the run must fit
+            bool ok = true;
+            uint64_t k = 0;
+#pragma unroll
+            for (int L = 1; L <= OD_NGRAM_MAX; ++L) {
+                int32_t id = (s + L - 1 < K) ? s_ids[s + L - 1] : -1;
+                ok = ok && (s + L <= K) && id >= 0 && id < v_q;
+                k |= (uint64_t)(uint32_t)(id + 1) << (16 * (L - 1));
+                valid[L] = ok && L >= 2;
+                key[L] = k;
+                grp[L] = od_hash64(k) & (ngroups - 1);
+            }
+#pragma unroll
+            for (int L = 2; L <= OD_NGRAM_MAX; ++L)
+                kl[L] = valid[L] ? __ldg(keys + grp[L] * OD_GROUP + lane) : 0ULL;
+#pragma unroll
+            for (int L = 2; L <= OD_NGRAM_MAX; ++L)
+                if (valid[L]) hit[L] = probe_continue(keys, vals, ngroups, key[L], grp[L], kl[L], lane);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int L = 2; L <= OD_NGRAM_MAX; ++L) s_hit[s][L] = hit[L];
+        }
+    }
+    __syncthreads();
+
+    if (threadIdx.x == 0) {
+        const size_t o = (size_t)b * K_max;
+        int pos = 0, m = 0;
+        uint32_t hits = 0, invalid = 0;
+        uint8_t tail = OD_TAIL_COMPLETE;
+        while (pos < K) {
+            int L = 0;
+            int32_t t = -1;
+            for (int len = OD_NGRAM_MAX; len >= 2; --len)
+                if (pos + len <= K && s_hit[pos][len] >= 0) { L = len; t = s_hit[pos][len]; break; }
+            if (L) {
+                float prod = q_sel[o + pos];
+                for (int j = 1; j < L; ++j) prod *= q_sel[o + pos + j];
+                tgt_ids[o + m] = t; q_prime[o + m] = prod;
+                span_start[o + m] = pos; span_len[o + m] = L;
+                ++m; pos += L; ++hits;
+                continue;
+            }
+            const int32_t id = s_ids[pos];
+            const bool in_vocab = id >= 0 && id < v_q;
+            if (!in_vocab) ++invalid;
+            const int32_t direct = in_vocab ? __ldg(vocab_map + id) : -1;
+            if (direct >= 0) {
+                tgt_ids[o + m] = direct; q_prime[o + m] = q_sel[o + pos];
+                span_start[o + m] = pos; span_len[o + m] = 1;
+                ++m; ++pos;
+            } else {
+                span_start[o + m] = pos; span_len[o + m] = 1;
+                tail = OD_TAIL_UNMAPPED_STOP;
+                break;
+            }
+        }
+        m_out[b] = m;
+        tail_kind[b] = tail;
+        if (counters) {
+            if (hits) atomicAdd(counters + OD_CNT_CACHE_HITS, hits);
+            if (tail == OD_TAIL_UNMAPPED_STOP) atomicAdd(counters + OD_CNT_UNMAPPED_STOPS, 1u);
+            if (invalid) atomicAdd(counters + OD_CNT_INVALID_IDS, invalid);
+            if (m) atomicAdd(counters + OD_CNT_MAPPED_TOKENS, (uint32_t)m);
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids,
+                          const int32_t *draft_len, const float *q_sel, int32_t *tgt_ids,
+                          float *q_prime, int32_t *span_start, int32_t *span_len, int32_t *m,
+                          uint8_t *tail_kind, uint32_t *counters, cudaStream_t s)
+{
+    if (B == 0) return cudaSuccess;
+    const int threads = K_max * OD_WARP;
+    od_map_kernel<<<B, threads, 0, s>>>(B, K_max, c->v_q, draft_ids, draft_len, q_sel,
+                                        c->d_vocab_map, c->d_keys, c->d_vals, c->cap, tgt_ids,
+                                        q_prime, span_start, span_len, m, tail_kind, counters);
+    return cudaGetLastError();
+}
