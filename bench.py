@@ -1,0 +1,425 @@
+#!/usr/bin/env python
+"""Benchmark of the cross-vocabulary verification step (one JSON line).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+A step is one pass of the whole hot path (od_map_proposals -> od_verify ->
+od_sample_residual) over one batch of synthetic input. The default workload is
+the batched 128256-id configuration (config 4); steps cycle through a pool of
+distinct input buffers larger than the L2 so every step's logits come from HBM.
+The K timed steps are captured into one CUDA graph (the kernels run back to back
+as in a decode loop) and timed with CUDA events between a barrier +
+synchronize on both sides; with N > 1 every rank runs its own full batch (weak
+scaling, no data-path collective) and the time is the max over ranks.
+
+Also reported: `roofline` for od_verify (algorithmic logit bytes / its own
+average launch duration from a graph of the same K launches, against the
+measured HBM copy rate), `e2e` (the same metric through od_step_host with pinned
+host buffers, copies inside the timed region), `cpu_baseline` (the CPU oracle as
+it stands on a bounded sample), and the SM clocks seen during the timed region.
+
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "verified_draft_tokens_per_sec"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4)
+    ap.add_argument("--pool", type=int, default=0, help="distinct step buffers (0 = enough for 4x L2)")
+    ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--verify-chunk-bytes", type=int, default=0)
+    ap.add_argument("--sample-tiles-per-block", type=int, default=0)
+    return ap.parse_args()
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def ncu_traffic(workload: str):
+    """Per-launch DRAM bytes of od_verify from the committed ncu summary, if any."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(p) as f:
+            return json.load(f).get(workload)
+    except Exception:
+        return None
+
+
+def step_bytes(s):
+    t = (s.draft_ids, s.draft_len, s.q_sel, s.q_rows, s.logits, s.temperature, s.seed)
+    return sum(x.numel() * x.element_size() for x in t)
+
+
+def oracle_time(w, st, steps, seconds):
+    """Oracle on host cores, one full batch per step, until `seconds` have passed
+    (at least one step). Returns (tokens, elapsed_s, steps_done, threads)."""
+    import oracle
+    from paper_2507_02659_b200 import synth
+    cache = oracle.Cache(st.runs, st.run_len, st.run_target)
+    threads = oracle.max_threads()
+    tokens, elapsed, done = 0, 0.0, 0
+    for i in range(steps):
+        s = synth.make_step(w, st, i, device="cpu")
+        lg, code = oracle.logits_to_numpy(s.logits)
+        args = (cache, st.vocab_map, w.v_p, s.draft_ids.numpy(), s.draft_len.numpy(), s.q_sel.numpy(),
+                s.q_rows.numpy(), lg, code, s.temperature.numpy(), s.seed.numpy().astype(np.uint64), i)
+        t0 = time.perf_counter()
+        oracle.step_batch(*args, threads=threads)
+        elapsed += time.perf_counter() - t0
+        tokens += int(s.draft_len.sum())
+        done += 1
+        if elapsed >= seconds:
+            break
+    return tokens, elapsed, done, threads
+
+
+def run_reference(a):
+    """The CPU oracle as the reference arm: rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2507_02659_b200 import synth
+    w = synth.paper_config(a.config)
+    st = synth.make_static(w)
+    # one step = a bounded sample of the workload: the first sequences of a batch
+    sel = min(w.B, 16)
+    w_s = synth.scaled(w, B=sel)
+    import oracle
+    cache = oracle.Cache(st.runs, st.run_len, st.run_target)
+    threads = oracle.max_threads()
+    steps = []
+    for i in range(a.warmup + a.steps):
+        s = synth.make_step(w_s, st, i, device="cpu")
+        lg, code = oracle.logits_to_numpy(s.logits)
+        steps.append((s, lg, code))
+        if len(steps) >= 8:
+            break
+    tokens, t_total = 0, 0.0
+    for i in range(a.warmup + a.steps):
+        s, lg, code = steps[i % len(steps)]
+        t0 = time.perf_counter()
+        oracle.step_batch(cache, st.vocab_map, w.v_p, s.draft_ids.numpy(), s.draft_len.numpy(),
+                          s.q_sel.numpy(), s.q_rows.numpy(), lg, code, s.temperature.numpy(),
+                          s.seed.numpy().astype(np.uint64), i, threads=threads)
+        dt = time.perf_counter() - t0
+        if i >= a.warmup:
+            t_total += dt
+            tokens += int(s.draft_len.sum())
+    value = tokens / t_total
+    sample = f"{sel} of {w.B} sequences per step, {a.steps} steps"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": a.gpus,
+        "steps": a.steps, "warmup": a.warmup, "ms_per_step": 1e3 * t_total / a.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "B": sel, "k_max": w.k_max,
+                                         "draft_vocab": w.v_q, "target_vocab": w.v_p,
+                                         "logit_dtype": w.logit_dtype},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    a = parse()
+    if a.impl == "reference":
+        return run_reference(a)
+    if a.warmup < 3:
+        a.warmup = 3
+
+    import torch.distributed as dist
+    from paper_2507_02659_b200 import binding as od
+    from paper_2507_02659_b200 import shard, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w0 = synth.paper_config(a.config)
+    w = shard.weak_shard(w0, rank, world)
+    st = synth.make_static(w)
+    ctx = od.Context(dev, w.v_q, w.v_p, w.B, w.k_max)
+    ctx.set_vocab_map(st.vocab_map)
+    ctx.cache_build(st.runs, st.run_len, st.run_target)
+    if a.verify_chunk_bytes:
+        ctx.set_option("verify_chunk_bytes", a.verify_chunk_bytes)
+    if a.sample_tiles_per_block:
+        ctx.set_option("sample_tiles_per_block", a.sample_tiles_per_block)
+
+    # pool of distinct step buffers, > 4x L2 in logits so no step finds its rows in L2
+    s0 = synth.make_step(w, st, 0, device=dev)
+    logit_bytes = s0.logits.numel() * s0.logits.element_size()
+    P = a.pool or max(3, -(-4 * L2_BYTES // logit_bytes))
+    P = min(P, a.steps + a.warmup)
+    pool = [s0] + [synth.make_step(w, st, i, device=dev) for i in range(1, P)]
+    B, K = w.B, w.k_max
+    esz = s0.logits.element_size()
+    mps = [od.alloc_map_out(ctx, B, K) for _ in range(P)]
+    vos = [od.alloc_verify_out(ctx, B, K) for _ in range(P)]
+    sos = [od.alloc_sample_out(ctx, B) for _ in range(P)]
+
+    def k1(i, step):
+        s = pool[i]
+        od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel, out=mps[i])
+
+    def k2(i, step):
+        s = pool[i]
+        od.od_verify(ctx, s.logits, mps[i], s.temperature, s.seed, step, out=vos[i])
+
+    def k3(i, step):
+        s = pool[i]
+        od.od_sample_residual(ctx, s.logits, vos[i], s.q_rows, s.draft_ids, mps[i], s.temperature,
+                              s.seed, step, out=sos[i])
+
+    def full_step(step):
+        i = step % P
+        k1(i, step); k2(i, step); k3(i, step)
+
+    # warm-up (also fills m for the K2-only graph)
+    for step in range(a.warmup):
+        full_step(step)
+    for i in range(P):
+        k1(i, 0)
+    torch.cuda.synchronize(dev)
+    rows_per_slot = [int((mps[i].m.clamp(0, K) + 1).sum().item()) for i in range(P)]
+    tokens_per_slot = [int(pool[i].draft_len.sum().item()) for i in range(P)]
+
+    def make_graph(fn, n, first):
+        if a.no_graph:
+            return None
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for k in range(n):
+                fn(first + k)
+        return g
+
+    g_step = make_graph(full_step, a.steps, a.warmup)
+    g_k2 = make_graph(lambda step: k2(step % P, step), a.steps, a.warmup)
+    g_k3 = make_graph(lambda step: k3(step % P, step), a.steps, a.warmup)
+    g_k1 = make_graph(lambda step: k1(step % P, step), a.steps, a.warmup)
+
+    def timed(g, fn):
+        """ms for the K steps, device-timed between barrier + synchronize."""
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        if g is not None:
+            g.replay()
+        else:
+            for k in range(a.steps):
+                fn(a.warmup + k)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        return e0.elapsed_time(e1)
+
+    # one untimed replay of each graph, then the timed region
+    for g in (g_step, g_k2, g_k3, g_k1):
+        if g is not None:
+            g.replay()
+    torch.cuda.synchronize(dev)
+    clocks = ClockSampler(local)
+    if rank == 0:
+        clocks.start()
+        time.sleep(0.3)
+    ms_step = timed(g_step, full_step)
+    # repeats of the same K steps: more samples of the clocks under this load, and a
+    # check that the first timed region was not an outlier
+    extra, t_end = [], time.perf_counter() + 1.5
+    while time.perf_counter() < t_end and len(extra) < 400:
+        extra.append(timed(g_step, full_step))
+    ms_k2 = timed(g_k2, lambda step: k2(step % P, step))
+    ms_k3 = timed(g_k3, lambda step: k3(step % P, step))
+    ms_k1 = timed(g_k1, lambda step: k1(step % P, step))
+    clk = clocks.stop() if rank == 0 else None
+
+    steps_idx = [(a.warmup + k) % P for k in range(a.steps)]
+    tokens_local = sum(tokens_per_slot[i] for i in steps_idx)
+    rows_total = sum(rows_per_slot[i] for i in steps_idx)
+    ms_max, tokens_all = shard.reduce_timing(ms_step, tokens_local, dev)
+    value = tokens_all / (ms_max * 1e-3)
+
+    k2_bytes_per_launch = rows_total * w.v_p * esz / a.steps
+    k2_ms_per_launch = ms_k2 / a.steps
+    achieved = k2_bytes_per_launch / (k2_ms_per_launch * 1e-3) / 1e9
+    peak, peak_src = measured_peak()
+
+    # end to end through od_step_host: pinned host inputs, copies inside the timed region
+    e2e = None
+    if not a.no_e2e:
+        ctx.host_step_reserve(od.OD_BF16 if w.logit_dtype == "bf16" else od.OD_F32)
+        hp = min(2, P)
+        hosts = []
+        for i in range(hp):
+            h = pool[i].to("cpu")
+            hosts.append(synth.StepInputs(*[t.contiguous().pin_memory() for t in
+                                            (h.draft_ids, h.draft_len, h.q_sel, h.q_rows, h.logits,
+                                             h.temperature, h.seed)], h.step))
+        hout = od.alloc_host_step_out(B, K)
+        n_e = max(1, a.e2e_steps)
+
+        def host_step(k):
+            h = hosts[k % hp]
+            od.od_step_host(ctx, h.draft_ids, h.draft_len, h.q_sel, h.q_rows, h.logits, h.temperature,
+                            h.seed, k, out=hout)
+        for k in range(3):
+            host_step(k)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for k in range(n_e):
+            host_step(k)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms_e = e0.elapsed_time(e1)
+        tok_e = sum(int(hosts[k % hp].draft_len.sum()) for k in range(n_e))
+        ms_e_max, tok_e_all = shard.reduce_timing(ms_e, tok_e, dev)
+        d2h = sum(t.numel() * t.element_size() for t in
+                  (hout.n_accepted, hout.n_draft_accepted, hout.out_token, hout.tgt_ids, hout.m,
+                   hout.verify_flags, hout.sample_flags))
+        e2e = {"value": tok_e_all / (ms_e_max * 1e-3), "unit": UNIT, "steps": n_e,
+               "ms_per_step": ms_e_max / n_e, "h2d_bytes_per_step": step_bytes(hosts[0]),
+               "d2h_bytes_per_step": d2h, "api": "od_step_host (pinned host buffers)"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not a.no_cpu_baseline:
+        nseq = min(w.B, 64)
+        tok, el, done, threads = oracle_time(synth.scaled(w, B=nseq), st, 64, a.cpu_seconds)
+        cpu = {"value": tok / el, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"{done} steps of {nseq} of the batch's {w.B} sequences ({el:.1f} s of oracle time)"}
+
+    if rank == 0:
+        acc = sum(int(vos[i].n_accepted.sum().item()) for i in range(P))
+        prop = sum(tokens_per_slot)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps,
+            "warmup": a.warmup, "ms_per_step": ms_max / a.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w0.name, "B_per_gpu": w.B, "k_max": w.k_max, "draft_vocab": w.v_q,
+                       "target_vocab": w.v_p, "logit_dtype": w.logit_dtype,
+                       "cache_entries": w.cache_entries, "pool_buffers": P,
+                       "l2_policy": f"inputs larger than L2: {P} distinct step buffers, "
+                                    f"{P * logit_bytes / 2**20:.0f} MiB of logits cycled",
+                       "launch": "K steps captured in one CUDA graph" if not a.no_graph else "eager launches",
+                       "parallelism": f"batch sharding x{world}, no collective"},
+            "gpu_launches": 3 * a.steps,
+            "kernels_ms_per_step": {"od_map_proposals": ms_k1 / a.steps, "od_verify": ms_k2 / a.steps,
+                                    "od_sample_residual": ms_k3 / a.steps,
+                                    "step_repeats": len(extra),
+                                    "step_repeat_median_ms": (statistics.median(extra) / a.steps) if extra else None},
+            "roofline": {"kernel": "od_verify", "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                         "bytes_per_launch": k2_bytes_per_launch,
+                         "us_per_launch": 1e3 * k2_ms_per_launch,
+                         "frac_of_theoretical_8184": achieved / 8184.0,
+                         "traffic": ncu_traffic(w0.name)},
+            "e2e": e2e, "cpu_baseline": cpu, "clocks": clk,
+            "stats": {"acceptance_rate": acc / max(1, prop), "rows_per_step": rows_total / a.steps,
+                      "draft_tokens_per_step": tokens_local / a.steps,
+                      "verify_grid": ctx.last_launch_info(0), "verify_chunk_elems": ctx.last_launch_info(1),
+                      "sample_grid": ctx.last_launch_info(2)},
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
