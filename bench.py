@@ -57,8 +57,9 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--verify-chunk-bytes", type=int, default=0)
-    ap.add_argument("--sample-tiles-per-block", type=int, default=0)
+    ap.add_argument("--verify-blocks-per-sm", type=int, default=0)
+    ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
+    ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches")
     return ap.parse_args()
 
 
@@ -233,10 +234,12 @@ def main():
     ctx = od.Context(dev, w.v_q, w.v_p, w.B, w.k_max)
     ctx.set_vocab_map(st.vocab_map)
     ctx.cache_build(st.runs, st.run_len, st.run_target)
-    if a.verify_chunk_bytes:
-        ctx.set_option("verify_chunk_bytes", a.verify_chunk_bytes)
-    if a.sample_tiles_per_block:
-        ctx.set_option("sample_tiles_per_block", a.sample_tiles_per_block)
+    if a.verify_blocks_per_sm:
+        ctx.set_option("verify_blocks_per_sm", a.verify_blocks_per_sm)
+    if a.sample_tiles_per_warp:
+        ctx.set_option("sample_tiles_per_warp", a.sample_tiles_per_warp)
+    if a.no_pdl:
+        ctx.set_option("pdl", 0)
 
     # pool of distinct step buffers, > 4x L2 in logits so no step finds its rows in L2
     s0 = synth.make_step(w, st, 0, device=dev)
@@ -413,7 +416,7 @@ def main():
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clk,
             "stats": {"acceptance_rate": acc / max(1, prop), "rows_per_step": rows_total / a.steps,
                       "draft_tokens_per_step": tokens_local / a.steps,
-                      "verify_grid": ctx.last_launch_info(0), "verify_chunk_elems": ctx.last_launch_info(1),
+                      "verify_grid": ctx.last_launch_info(0), "verify_span_a": ctx.last_launch_info(1),
                       "sample_grid": ctx.last_launch_info(2)},
         }
         print(json.dumps(out))

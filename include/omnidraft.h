@@ -130,9 +130,12 @@ int32_t od_cache_build(od_ctx *ctx, const int32_t *host_runs,
                        const int32_t *host_len, const int32_t *host_target,
                        int64_t E);
 
-/* Tuning knobs, mainly for experiments. Names: "verify_chunk_bytes" (bytes of
- * one logit row given to one thread block, 0 = automatic), "sample_tiles_per_block"
- * (0 = automatic). Unknown name: INVALID_ARG. */
+/* Tuning knobs, mainly for experiments. Names: "verify_blocks_per_sm" (thread
+ * blocks of od_verify per multiprocessor, 1..8, 0 = automatic),
+ * "sample_tiles_per_warp" (256-id tiles one warp of od_sample_residual sums,
+ * 0 = automatic), "pdl" (1 = launch the step kernels with programmatic stream
+ * serialization so that a kernel's prologue overlaps its predecessor's tail,
+ * the default; 0 = plain stream order). Unknown name: INVALID_ARG. */
 int32_t od_set_option(od_ctx *ctx, const char *name, int64_t value);
 
 /* ---- the step ----------------------------------------------------------- */
@@ -241,10 +244,9 @@ int32_t od_step_host(od_ctx *ctx, int32_t B, int32_t K_max,
 
 /* ---- misc ---------------------------------------------------------------- */
 
-/* Number of thread blocks the last od_verify / od_sample_residual call on this
- * context launched and the bytes of one row chunk (for benchmarks). which: 0 =
- * verify grid size, 1 = verify chunk elements, 2 = sample grid size, 3 = sample
- * tiles per block. */
+/* Launch shape of the last od_verify / od_sample_residual call on this context
+ * (for benchmarks). which: 0 = verify grid size, 1 = 512-byte units of row 0
+ * data per warp, 2 = sample grid size, 3 = sample tiles per warp. */
 int64_t od_last_launch_info(const od_ctx *ctx, int32_t which);
 
 const char *od_status_string(int32_t status);

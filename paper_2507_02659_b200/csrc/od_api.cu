@@ -44,7 +44,7 @@ int32_t dev_alloc(T **p, size_t n)
 void free_all(od_ctx *c)
 {
     void *ptrs[] = {c->d_vocab_map, c->d_inv_map, c->d_keys, c->d_vals, c->d_partials,
-                    c->d_row_ticket, c->d_seq_ticket, c->d_seq_bits, c->d_tile_sums,
+                    c->d_tile_sums,
                     c->d_samp_ticket, c->s_logits, c->s_q_rows, c->s_q_sel, c->s_temperature,
                     c->s_draft_ids, c->s_draft_len, c->s_seed, c->s_tgt_ids, c->s_span_start,
                     c->s_span_len, c->s_m, c->s_n_acc, c->s_n_draft, c->s_token, c->s_q_prime,
@@ -104,17 +104,15 @@ int32_t od_create(od_ctx **ctx, int32_t device, int32_t draft_vocab, int32_t tar
         delete c;
         return OD_ERR_CUDA;
     }
-    // a row is never cut finer than 4 KB (fp32 rows are the longest in bytes)
-    c->max_chunks = (int32_t)(((int64_t)target_vocab * 4 + 4095) / 4096);
+    c->opt_pdl = 1;
     c->tiles_per_row = (target_vocab + OD_SAMPLE_TILE - 1) / OD_SAMPLE_TILE;
-    const size_t rows = (size_t)max_batch * (max_k + 1);
+    // od_verify scratch serves one launch: at most OD_VERIFY_MAX_B sequences
+    const size_t vb = max_batch < OD_VERIFY_MAX_B ? max_batch : OD_VERIFY_MAX_B;
+    const size_t rows = vb * (max_k + 1);
     int32_t st = OD_OK;
     if (st == OD_OK) st = dev_alloc(&c->d_vocab_map, (size_t)draft_vocab);
     if (st == OD_OK) st = dev_alloc(&c->d_inv_map, (size_t)target_vocab + 8);
-    if (st == OD_OK) st = dev_alloc(&c->d_partials, rows * c->max_chunks);
-    if (st == OD_OK) st = dev_alloc(&c->d_row_ticket, rows);
-    if (st == OD_OK) st = dev_alloc(&c->d_seq_ticket, (size_t)max_batch);
-    if (st == OD_OK) st = dev_alloc(&c->d_seq_bits, (size_t)max_batch * 2);
+    if (st == OD_OK) st = dev_alloc(&c->d_partials, rows * OD_VERIFY_SEG_MAX);
     if (st == OD_OK) st = dev_alloc(&c->d_tile_sums, (size_t)max_batch * c->tiles_per_row);
     if (st == OD_OK) st = dev_alloc(&c->d_samp_ticket, (size_t)max_batch);
     if (st != OD_OK) {
@@ -222,8 +220,9 @@ int32_t od_cache_build(od_ctx *c, const int32_t *host_runs, const int32_t *host_
 int32_t od_set_option(od_ctx *c, const char *name, int64_t value)
 {
     if (!c || !name || value < 0) return OD_ERR_INVALID_ARG;
-    if (!strcmp(name, "verify_chunk_bytes")) { c->opt_verify_chunk_bytes = value; return OD_OK; }
-    if (!strcmp(name, "sample_tiles_per_block")) { c->opt_sample_tiles_per_block = value; return OD_OK; }
+    if (!strcmp(name, "verify_blocks_per_sm")) { c->opt_verify_blocks_per_sm = value; return OD_OK; }
+    if (!strcmp(name, "sample_tiles_per_warp")) { c->opt_sample_tiles_per_warp = value; return OD_OK; }
+    if (!strcmp(name, "pdl")) { c->opt_pdl = value != 0; return OD_OK; }
     return OD_ERR_INVALID_ARG;
 }
 

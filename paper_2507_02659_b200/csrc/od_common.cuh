@@ -10,9 +10,10 @@
 
 #define OD_WARP 32
 #define OD_GROUP 32                 // slots of one hash-table probe group
-#define OD_SAMPLE_TILE 2048         // elements of one residual-sampler tile
+#define OD_SAMPLE_TILE 256          // elements of one residual-sampler tile (8 per lane of a warp)
 #define OD_SAMPLE_THREADS 256
-#define OD_VERIFY_THREADS 256
+#define OD_VERIFY_SEG_MAX 64        // most segments (partials) one logit row is cut into
+#define OD_VERIFY_MAX_B 2048        // sequences per od_verify launch (longer batches go in slices)
 
 struct od_ctx {
     int device;
@@ -30,11 +31,7 @@ struct od_ctx {
     int64_t cap;                    // power of two, multiple of 32, or 0
 
     // od_verify scratch
-    float2 *d_partials;             // [max_batch*(max_k+1)*max_chunks] (max, sum)
-    unsigned int *d_row_ticket;     // [max_batch*(max_k+1)]
-    unsigned int *d_seq_ticket;     // [max_batch]
-    unsigned int *d_seq_bits;       // [max_batch][2]: accept bits | boundary bits << 16; misc
-    int32_t max_chunks;
+    float4 *d_partials;             // [rows][OD_VERIFY_SEG_MAX] (c, sum, max, -), rows of one launch
 
     // od_sample_residual scratch
     double *d_tile_sums;            // [max_batch * tiles_per_row]
@@ -42,8 +39,9 @@ struct od_ctx {
     int32_t tiles_per_row;
 
     // options
-    int64_t opt_verify_chunk_bytes;
-    int64_t opt_sample_tiles_per_block;
+    int64_t opt_verify_blocks_per_sm;
+    int64_t opt_sample_tiles_per_warp;
+    int64_t opt_pdl;                // launch with programmatic stream serialization
 
     // last launch info
     int64_t info[4];

@@ -44,6 +44,11 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
     __shared__ int32_t s_ids[OD_MAX_K];
     __shared__ int32_t s_hit[OD_MAX_K][OD_NGRAM_MAX + 1];   // [offset][length] -> target or -1
 
+    // under programmatic dependent launch: wait for everything earlier in the
+    // stream first, only then let the verification kernel start its prefetch
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+
     const int b = blockIdx.x;
     if (b >= B) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -137,9 +142,17 @@ cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *dr
                           uint8_t *tail_kind, uint32_t *counters, cudaStream_t s)
 {
     if (B == 0) return cudaSuccess;
-    const int threads = K_max * OD_WARP;
-    od_map_kernel<<<B, threads, 0, s>>>(B, K_max, c->v_q, draft_ids, draft_len, q_sel,
-                                        c->d_vocab_map, c->d_keys, c->d_vals, c->cap, tgt_ids,
-                                        q_prime, span_start, span_len, m, tail_kind, counters);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)B);
+    cfg.blockDim = dim3((unsigned)(K_max * OD_WARP));
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->opt_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, od_map_kernel, B, K_max, c->v_q, draft_ids, draft_len, q_sel,
+                              (const int32_t *)c->d_vocab_map, (const uint64_t *)c->d_keys,
+                              (const int32_t *)c->d_vals, c->cap, tgt_ids, q_prime, span_start,
+                              span_len, m, tail_kind, counters);
 }

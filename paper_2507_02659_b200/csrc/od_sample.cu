@@ -4,14 +4,15 @@
 // paragraph of Section 3; Section 3.1, Eq. (2); Algorithm 1, rejection and
 // free-token lines).
 //
-// Inverse-CDF sampling in target-id order, organised as tiles of 2048 ids:
-//   pass 1  every block computes r(t) for its tiles of row j = n_b and stores
-//           one fp64 sum per tile;
+// Inverse-CDF sampling in target-id order over tiles of 256 ids (8 consecutive
+// ids per lane of one warp, so a tile needs shuffles only, no block barrier):
+//   pass 1  every warp computes r(t) for its run of tiles of row j = n_b and
+//           stores one fp64 sum per tile;
 //   ticket  blocks never wait for each other: the block that draws the
 //           sequence's last ticket continues alone;
-//   pass 2  that block scans the tile sums (R = total, target = u * R), finds
-//           the tile in which the running sum crosses the target, recomputes
-//           that one tile (2048 ids, L2-resident) and scans inside it.
+//   pass 2  that block scans the tile sums in parallel (R = total, target =
+//           u * R), finds the tile in which the running sum crosses the target,
+//           and one warp recomputes that tile (L2-resident) and scans inside it.
 // r(t) is evaluated in fp32 exactly the same way in both passes; all sums and
 // scans are fp64 in a fixed order, so the result is reproducible and the only
 // difference to exact arithmetic is the fp32 rounding of the individual r(t).
@@ -21,11 +22,14 @@
 
 namespace {
 
+constexpr int WARPS = OD_SAMPLE_THREADS / 32;
+constexpr int EPT = OD_SAMPLE_TILE / 32;                  // ids per lane per tile (8)
+
 struct SampleArgs {
     const void *logits;
     int64_t row_stride, seq_stride;
     int32_t B, K_max, v_p, v_q;
-    int32_t tiles_per_row, tiles_per_block;
+    int32_t ntiles, tiles_per_warp;
     const float *row_max, *row_sum, *q_rows;
     const int32_t *draft_ids, *tgt_ids;
     const float *q_prime;
@@ -43,7 +47,7 @@ struct SampleArgs {
     unsigned int *ticket;
 };
 
-// what one sequence's blocks need to evaluate r(t)
+// what one sequence's warps need to evaluate r(t)
 struct SeqState {
     const char *row;
     const float *q_row;
@@ -53,13 +57,9 @@ struct SeqState {
     float ngram_prob, prefix_val;
 };
 
-constexpr int EPT = OD_SAMPLE_TILE / OD_SAMPLE_THREADS;   // elements per thread per tile (8)
-
-template <int DTYPE>
-__device__ __forceinline__ float r_of(const SeqState &q, const int32_t *__restrict__ inv_map,
-                                      bool residual, int64_t t, float x, int32_t d)
+__device__ __forceinline__ float r_of(const SeqState &q, bool residual, int64_t t, float x, int32_t d)
 {
-    float p = od_ex2((x - q.M) * q.scale) * q.invS;
+    const float p = od_ex2((x - q.M) * q.scale) * q.invS;
     if (!residual) return p;
     float qq = d >= 0 ? __ldg(q.q_row + d) : 0.f;
     if (t == q.prefix_token) qq = q.prefix_val;
@@ -67,15 +67,15 @@ __device__ __forceinline__ float r_of(const SeqState &q, const int32_t *__restri
     return fmaxf(0.f, p - qq);
 }
 
-// r(t) of the EPT consecutive ids a thread owns in `tile`; ids >= v_p give 0
+// r(t) of the EPT consecutive ids this lane owns in `tile`; ids >= v_p give 0
 template <int DTYPE>
 __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs &a, bool residual,
-                                            int tile, float *r)
+                                            int tile, int lane, float *r)
 {
-    const int64_t t0 = (int64_t)tile * OD_SAMPLE_TILE + (int64_t)threadIdx.x * EPT;
-    float x[EPT];
-    int32_t d[EPT];
+    const int64_t t0 = (int64_t)tile * OD_SAMPLE_TILE + (int64_t)lane * EPT;
     if (t0 + EPT <= a.v_p) {
+        float x[EPT];
+        int32_t d[EPT];
         if (DTYPE == OD_BF16) {
             const uint4 v = __ldg((const uint4 *)(q.row + (size_t)t0 * 2));
             x[0] = od_bf16_lo(v.x); x[1] = od_bf16_hi(v.x); x[2] = od_bf16_lo(v.y); x[3] = od_bf16_hi(v.y);
@@ -93,7 +93,7 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
             d[4] = i1.x; d[5] = i1.y; d[6] = i1.z; d[7] = i1.w;
         }
 #pragma unroll
-        for (int e = 0; e < EPT; ++e) r[e] = r_of<DTYPE>(q, a.inv_map, residual, t0 + e, x[e], residual ? d[e] : -1);
+        for (int e = 0; e < EPT; ++e) r[e] = r_of(q, residual, t0 + e, x[e], residual ? d[e] : -1);
     } else {
 #pragma unroll
         for (int e = 0; e < EPT; ++e) {
@@ -101,7 +101,7 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
             if (t < a.v_p) {
                 const float xv = od_load_logit<DTYPE>(q.row, t);
                 const int32_t dv = residual ? __ldg(a.inv_map + t) : -1;
-                r[e] = r_of<DTYPE>(q, a.inv_map, residual, t, xv, dv);
+                r[e] = r_of(q, residual, t, xv, dv);
             } else {
                 r[e] = 0.f;
             }
@@ -109,46 +109,60 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
     }
 }
 
-__device__ __forceinline__ double warp_sum(double v)
+__device__ __forceinline__ double lane_sum(const float *r)
 {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, off);
-    return v;
-}
-
-// sum of one tile, valid in thread 0; fixed order (index order inside a thread,
-// shuffle tree inside a warp, warps in order)
-template <int DTYPE>
-__device__ double tile_sum(const SeqState &q, const SampleArgs &a, bool residual, int tile,
-                           double *s_warp)
-{
-    float r[EPT];
-    tile_values<DTYPE>(q, a, residual, tile, r);
     double s = 0.0;
 #pragma unroll
     for (int e = 0; e < EPT; ++e) s += (double)r[e];
-    s = warp_sum(s);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    __syncthreads();
-    if (lane == 0) s_warp[warp] = s;
-    __syncthreads();
-    double tot = 0.0;
-    if (threadIdx.x == 0)
-        for (int w = 0; w < OD_SAMPLE_THREADS / 32; ++w) tot += s_warp[w];
-    return tot;
+    return s;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    return v;
+}
+
+// tile sums of tiles [t_lo, t_hi) by one warp: index order inside a lane, xor
+// tree across the lanes
+template <int DTYPE>
+__device__ __forceinline__ void warp_tiles(const SeqState &q, const SampleArgs &a, bool residual,
+                                           int t_lo, int t_hi, int lane, double *sums)
+{
+    int tile = t_lo;
+    for (; tile + 2 <= t_hi; tile += 2) {                  // two tiles in flight
+        float r0[EPT], r1[EPT];
+        tile_values<DTYPE>(q, a, residual, tile, lane, r0);
+        tile_values<DTYPE>(q, a, residual, tile + 1, lane, r1);
+        const double s0 = warp_sum(lane_sum(r0)), s1 = warp_sum(lane_sum(r1));
+        if (lane == 0) { sums[tile] = s0; sums[tile + 1] = s1; }
+    }
+    if (tile < t_hi) {
+        float r0[EPT];
+        tile_values<DTYPE>(q, a, residual, tile, lane, r0);
+        const double s0 = warp_sum(lane_sum(r0));
+        if (lane == 0) sums[tile] = s0;
+    }
+    __threadfence();                                       // the sums are read by another block
 }
 
 template <int DTYPE>
-__global__ void __launch_bounds__(OD_SAMPLE_THREADS)
+__global__ void __launch_bounds__(OD_SAMPLE_THREADS, 4)
 od_sample_kernel(const SampleArgs a)
 {
-    __shared__ double s_warp[OD_SAMPLE_THREADS / 32];
+    __shared__ double s_warp[WARPS];
     __shared__ unsigned int s_last;
-    __shared__ int s_tile, s_pick, s_lastpos;
-    __shared__ double s_before, s_total, s_target, s_lo, s_hi;
+    __shared__ int s_tile, s_lastmass;
+    __shared__ double s_before, s_total;
+
+    // n_accepted and the row statistics come from the verification kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
 
     const int b = blockIdx.y;
     const int K = a.K_max;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int mb = a.m[b];
     mb = mb < 0 ? 0 : (mb > K ? K : mb);
     int j = a.n_accepted[b];
@@ -188,15 +202,15 @@ od_sample_kernel(const SampleArgs a)
     }
 
     // ---- pass 1: one fp64 sum per tile ----
-    const int ntiles = a.tiles_per_row;
+    const int ntiles = a.ntiles;
     double *sums = a.tile_sums + (size_t)b * ntiles;
-    const int t_lo = blockIdx.x * a.tiles_per_block;
-    int t_hi = t_lo + a.tiles_per_block;
-    if (t_hi > ntiles) t_hi = ntiles;
-    for (int tile = t_lo; tile < t_hi; ++tile) {
-        const double s = tile_sum<DTYPE>(q, a, q.residual, tile, s_warp);
-        if (threadIdx.x == 0) sums[tile] = s;
+    {
+        const int t_lo = (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
+        int t_hi = t_lo + a.tiles_per_warp;
+        if (t_hi > ntiles) t_hi = ntiles;
+        if (t_lo < t_hi) warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, sums);
     }
+    __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
@@ -209,103 +223,120 @@ od_sample_kernel(const SampleArgs a)
     bool residual = q.residual;
     uint32_t flags = residual ? 0u : OD_SF_BONUS;
     const float u = od_uniform(a.seed[b], a.step, (uint32_t)j, 1u);
+    const int per = (ntiles + OD_SAMPLE_THREADS - 1) / OD_SAMPLE_THREADS;
+    const int my_lo = threadIdx.x * per;
+    const int my_hi = my_lo + per < ntiles ? my_lo + per : ntiles;
+    const volatile double *vs = sums;
+    double target = 0.0;
     for (int attempt = 0; attempt < 2; ++attempt) {
-        if (threadIdx.x == 0) {
-            const volatile double *vs = sums;
-            double tot = 0.0;
-            for (int t = 0; t < ntiles; ++t) tot += vs[t];
-            s_total = tot;
-            s_tile = -1;
-            if (tot > 0.0) {
-                const double target = (double)u * tot;
-                double c = 0.0, before = 0.0;
-                int pick = -1;
-                for (int t = 0; t < ntiles; ++t) {          // same order as the total above
-                    const double nc = c + vs[t];
-                    if (nc > target) { pick = t; before = c; break; }
-                    c = nc;
-                }
-                if (pick < 0) {                             // unreachable for u < 1; stay safe
-                    c = 0.0;
-                    for (int t = 0; t < ntiles; ++t) {
-                        if (vs[t] > 0.0) { pick = t; before = c; }
-                        c += vs[t];
-                    }
-                }
-                s_tile = pick; s_before = before; s_target = target;
+        // exclusive scan of the tile sums: thread i owns `per` consecutive tiles
+        double loc = 0.0;
+        for (int t = my_lo; t < my_hi; ++t) loc += vs[t];
+        double inc = loc;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const double v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+            if (lane >= off) inc += v;
+        }
+        if (lane == 31) s_warp[warp] = inc;
+        if (threadIdx.x == 0) { s_tile = 0x7FFFFFFF; s_lastmass = -1; }
+        __syncthreads();
+        double base = 0.0;
+        for (int w = 0; w < warp; ++w) base += s_warp[w];
+        if (threadIdx.x == OD_SAMPLE_THREADS - 1) s_total = base + inc;
+        __syncthreads();
+        const double R = s_total;
+        if (R > 0.0) {
+            target = (double)u * R;
+            double c = base + inc - loc;
+            int last = -1;
+            for (int t = my_lo; t < my_hi; ++t) {
+                const double v = vs[t];
+                if (v > 0.0) last = t;
+                if (c + v > target) { atomicMin(&s_tile, t); break; }   // first crossing of this run
+                c += v;
             }
-            s_pick = 0x7FFFFFFF; s_lastpos = -1;
+            if (last >= 0) atomicMax(&s_lastmass, last);
         }
         __syncthreads();
-        if (s_tile >= 0) break;
-        if (attempt == 1) break;
+        if (R > 0.0) {
+            // cumulative sums never decrease, so the smallest reported tile is the crossing;
+            // if rounding hid it, take the last tile that has mass
+            const int t_pick = s_tile != 0x7FFFFFFF ? s_tile : s_lastmass;
+            __syncthreads();
+            if (t_pick >= my_lo && t_pick < my_hi) {        // its owner publishes the sum before it
+                double c = base + inc - loc;
+                for (int t = my_lo; t < t_pick; ++t) c += vs[t];
+                s_before = c;
+                s_tile = t_pick;
+            }
+            __syncthreads();
+            break;
+        }
+        if (attempt == 1) {
+            if (threadIdx.x == 0) s_tile = -1;
+            __syncthreads();
+            break;
+        }
         // no residual mass: draw from p_j instead (rare; this block redoes the row)
         residual = false;
         flags |= OD_SF_ZERO_MASS;
-        for (int tile = 0; tile < ntiles; ++tile) {
-            const double s = tile_sum<DTYPE>(q, a, false, tile, s_warp);
-            if (threadIdx.x == 0) sums[tile] = s;
-        }
+        for (int t_lo = warp * 2; t_lo < ntiles; t_lo += WARPS * 2)
+            warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 2 < ntiles ? t_lo + 2 : ntiles, lane, sums);
         __syncthreads();
     }
-    if (s_tile < 0) {                               // no mass at all (non-finite input)
+    if (s_tile < 0 || s_tile == 0x7FFFFFFF) {       // no mass at all (non-finite input)
         if (threadIdx.x == 0) {
             a.out_token[b] = -1; a.resid_mass[b] = (float)s_total; a.flags[b] = flags | OD_SF_ZERO_MASS;
             a.ticket[b] = 0;
         }
         return;
     }
+    if (warp != 0) return;
 
-    // scan inside the chosen tile
+    // ---- warp 0 scans inside the chosen tile ----
     const int tile = s_tile;
+    const double R = s_total;
     float r[EPT];
-    tile_values<DTYPE>(q, a, residual, tile, r);
-    double mine = 0.0;
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) mine += (double)r[e];
-    // exclusive scan of the per-thread sums in thread order
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    tile_values<DTYPE>(q, a, residual, tile, lane, r);
+    const double mine = lane_sum(r);
     double incl = mine;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
         const double v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
         if (lane >= off) incl += v;
     }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    double base = s_before;
-    for (int w = 0; w < warp; ++w) base += s_warp[w];
-    double c = base + (incl - mine);
-    const double target = s_target;
-    const int64_t t0 = (int64_t)tile * OD_SAMPLE_TILE + (int64_t)threadIdx.x * EPT;
-    int my_pick = -1, my_last = -1;
+    double c = s_before + (incl - mine);
+    const int64_t t0 = (int64_t)tile * OD_SAMPLE_TILE + (int64_t)lane * EPT;
+    int my_pick = 0x7FFFFFFF, my_last = -1;
     double lo = 0.0, hi = 0.0;
 #pragma unroll
     for (int e = 0; e < EPT; ++e) {
         const double nc = c + (double)r[e];
         if (r[e] > 0.f) my_last = (int)(t0 + e);
-        if (my_pick < 0 && nc > target) { my_pick = (int)(t0 + e); lo = c; hi = nc; }
+        if (my_pick == 0x7FFFFFFF && nc > target) { my_pick = (int)(t0 + e); lo = c; hi = nc; }
         c = nc;
     }
-    if (my_pick >= 0) atomicMin(&s_pick, my_pick);
-    if (my_last >= 0) atomicMax(&s_lastpos, my_last);
-    __syncthreads();
-    if (my_pick >= 0 && my_pick == s_pick) { s_lo = lo; s_hi = hi; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int tok;
-        const double R = s_total;
-        if (s_pick != 0x7FFFFFFF) {
-            tok = s_pick;
-            const double margin = fmin(target - s_lo, s_hi - target);
+    int pick = my_pick, last = my_last;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        pick = min(pick, __shfl_xor_sync(0xFFFFFFFFu, pick, off));
+        last = max(last, __shfl_xor_sync(0xFFFFFFFFu, last, off));
+    }
+    if (pick != 0x7FFFFFFF) {
+        if (my_pick == pick) {                      // exactly one lane owns the picked id
+            const double margin = fmin(target - lo, hi - target);
             if (margin <= OD_TAU_SAMPLE * R) flags |= OD_SF_BOUNDARY;
-        } else {
-            tok = s_lastpos;                        // rounding: target beyond the tile's last edge
-            flags |= OD_SF_BOUNDARY;
+            a.out_token[b] = pick;
+            a.resid_mass[b] = (float)R;
+            a.flags[b] = flags;
+            a.ticket[b] = 0;
         }
-        a.out_token[b] = tok;
+    } else if (lane == 0) {
+        // rounding: target beyond the tile's last edge
+        a.out_token[b] = last;
         a.resid_mass[b] = (float)R;
-        a.flags[b] = flags;
+        a.flags[b] = flags | OD_SF_BOUNDARY | (last < 0 ? OD_SF_ZERO_MASS : 0u);
         a.ticket[b] = 0;
     }
 }
@@ -325,20 +356,21 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
 {
     if (B == 0) return cudaSuccess;
     const int ntiles = c->tiles_per_row;
-    int64_t tpb = c->opt_sample_tiles_per_block;
-    if (tpb <= 0) {
-        // aim at ~8 blocks per SM over the whole batch
-        const int64_t want = (int64_t)c->sm_count * 8;
-        const int64_t per_row = (want + B - 1) / B;
-        tpb = (ntiles + per_row - 1) / per_row;
-        if (tpb < 1) tpb = 1;
+    int64_t tpw = c->opt_sample_tiles_per_warp;
+    if (tpw <= 0) {
+        // one resident wave (four 256-thread blocks per SM) over the whole batch
+        const int64_t want = (int64_t)c->sm_count * 4;
+        int64_t per_row = want / B;
+        if (per_row < 1) per_row = 1;
+        tpw = (ntiles + per_row * WARPS - 1) / (per_row * WARPS);
+        if (tpw < 1) tpw = 1;
     }
-    if (tpb > ntiles) tpb = ntiles;
-    const int blocks_x = (int)((ntiles + tpb - 1) / tpb);
+    const int64_t tiles_per_block = tpw * WARPS;
+    const int blocks_x = (int)((ntiles + tiles_per_block - 1) / tiles_per_block);
     SampleArgs a;
     a.logits = logits; a.row_stride = row_stride; a.seq_stride = seq_stride;
     a.B = B; a.K_max = K_max; a.v_p = c->v_p; a.v_q = c->v_q;
-    a.tiles_per_row = ntiles; a.tiles_per_block = (int32_t)tpb;
+    a.ntiles = ntiles; a.tiles_per_warp = (int32_t)tpw;
     a.row_max = row_max; a.row_sum = row_sum; a.q_rows = q_rows;
     a.draft_ids = draft_ids; a.tgt_ids = tgt_ids; a.q_prime = q_prime;
     a.span_start = span_start; a.span_len = span_len; a.m = m; a.tail_kind = tail_kind;
@@ -346,12 +378,18 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
     a.vocab_map = c->d_vocab_map; a.inv_map = c->d_inv_map;
     a.out_token = out_token; a.resid_mass = resid_mass; a.flags = flags;
     a.tile_sums = c->d_tile_sums; a.ticket = c->d_samp_ticket;
-    dim3 grid((unsigned)blocks_x, (unsigned)B);
     c->info[2] = (int64_t)blocks_x * B;
-    c->info[3] = tpb;
-    if (dtype == OD_BF16)
-        od_sample_kernel<OD_BF16><<<grid, OD_SAMPLE_THREADS, 0, s>>>(a);
-    else
-        od_sample_kernel<OD_F32><<<grid, OD_SAMPLE_THREADS, 0, s>>>(a);
-    return cudaGetLastError();
+    c->info[3] = tpw;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks_x, (unsigned)B);
+    cfg.blockDim = dim3(OD_SAMPLE_THREADS);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->opt_pdl ? 1 : 0;
+    return dtype == OD_BF16 ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16>, a)
+                            : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32>, a);
 }

@@ -2,31 +2,60 @@
 // acceptance ratios and the accepted prefix (Algorithm 1, target-probability
 // and rejection-sampling lines; acceptance ratio of Section 3.1).
 //
-// The kernel is a single streaming pass over the logits: every element is read
-// from HBM exactly once with 128-bit loads. A row is cut into chunks; one
-// thread block reduces one chunk to a (max, sum exp) pair: per thread a
-// running pair whose maximum is refreshed once per 16-byte vector (one rescale
-// per vector, not per element), then a fixed shuffle tree over the warp and
-// over the block's warps. Blocks never wait on one another: a block publishes
-// its pair, takes a ticket on the row's counter, and the block that draws the
-// last ticket merges the row's pairs in chunk order, evaluates p(t_i), the
-// ratio, the uniform and the accept bit; the last row of a sequence (a second
-// ticket) turns the accept bits into the prefix length. Tickets and bit words
-// are reset by their last user, so every launch starts from zeros.
+// Two launches.
 //
-// The reduction order is fixed (no floating-point atomics): results are
-// bit-identical from run to run.
+// (1) od_verify_stream_kernel: one streaming pass in which every logit crosses
+// HBM exactly once (128-bit loads, four in flight per thread, four 256-thread
+// blocks per SM: one resident wave). The bytes are split evenly over the
+// blocks, whatever the mix of row counts. The unit of work is 512 contiguous
+// bytes of a row; a row has W units; the rows to read are laid end to end in
+// two flat index spaces and every block takes one contiguous span of each:
+//   space A  row 0 of every sequence. It is always read, so its split needs
+//            nothing from the device: a block asks the copy engine to pull its
+//            span into L2 (cp.async.bulk.prefetch) before it waits for the
+//            translation kernel (programmatic dependent launch) and before it
+//            builds the prefix sums of m, so HBM is busy during both;
+//   space B  rows 1..m_b, split by the prefix sums of m, which every block
+//            rebuilds in shared memory (at most 2048 sequences per launch).
+// A span is cut at row ends into segments; a block reduces a segment to one
+// partial (reference exponent c, sum of exp2(x*scale - c), exact maximum) and
+// stores it. No atomics, no fences, no block waits for another.
+//
+// (2) od_verify_decide_kernel: one block per sequence, one warp per row. Before
+// it waits for the stream kernel it loads what does not depend on it (m, T,
+// t_i, q'(t_i), x[t_i], the Philox uniforms); afterwards warp r merges the
+// partials of row r, evaluates p(t_i), the ratio and the accept bit, and thread
+// 0 turns the bits into the accepted prefix.
+//
+// Arithmetic: exp((x - M)/T) is evaluated as exp2(fma(x, s, -c)) with
+// s = log2(e)/T and c = fl(r*s) for a running reference r >= every element
+// absorbed so far (refreshed once per group of vectors, not per element). A
+// partial is carried relative to its own c, partials are merged in the scaled
+// domain, and the row sum relative to the exact maximum M is recovered at the
+// end as S_c * exp2(fma(-M, s, c)), which removes the rounding of c. M itself
+// is tracked separately (packed bf16x2 maxima for bf16 rows). The reduction
+// order is fixed by (m, grid): results are bit-identical from run to run.
 #include <float.h>
 
 #include "od_common.cuh"
 
 namespace {
 
+constexpr int THREADS = 256;
+constexpr int WARPS = THREADS / 32;
+constexpr int U = 4;                            // 16-byte loads in flight per thread
+#ifndef OD_VERIFY_BLOCKS_PER_SM
+#define OD_VERIFY_BLOCKS_PER_SM 4               // resident blocks per SM the register budget allows
+#endif
+
 struct VerifyArgs {
     const void *logits;
     int64_t row_stride, seq_stride;     // elements
     int32_t B, K_max, v_p;
-    int32_t chunk_elems, chunks;
+    int32_t W;                          // 512-byte units per row
+    int32_t n_chunks;                   // blocks of the stream grid
+    int32_t span_min;                   // keeps a row within OD_VERIFY_SEG_MAX segments
+    int32_t span_a;                     // units of space A per block
     const int32_t *tgt_ids;
     const float *q_prime;
     const int32_t *span_len;
@@ -37,41 +66,23 @@ struct VerifyArgs {
     float *row_max, *row_sum, *p_sel, *ratio;
     int32_t *n_accepted, *n_draft_accepted;
     uint32_t *flags;
-    float2 *partials;
-    unsigned int *row_ticket, *seq_ticket, *seq_bits;
+    float4 *partials;                   // [row slot][OD_VERIFY_SEG_MAX] (c, sum, max, -)
 };
 
-// running pair update with the 8 (bf16) or 4 (fp32) values of one vector
-__device__ __forceinline__ void absorb(float &m, float &s, const float *x, int n, float scale)
+// How many blocks hold pieces of flat row `rho` of a space whose blocks take
+// `span` units each.
+__device__ __forceinline__ int row_segments(uint32_t rho, uint32_t W, uint32_t span)
 {
-    float vm = x[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i)
-        if (i < n) vm = fmaxf(vm, x[i]);
-    if (vm > m) {
-        s *= od_ex2((m - vm) * scale);
-        m = vm;
-    }
-    float acc = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        if (i < n) acc += od_ex2((x[i] - m) * scale);
-    s += acc;
+    return (int)(((rho + 1) * W - 1) / span - rho * W / span + 1);
 }
 
-template <int DTYPE>
-__device__ __forceinline__ void unpack(const uint4 &v, float *x)
+__device__ __forceinline__ uint32_t span_of_space_b(uint32_t rows_b, uint32_t W, uint32_t n_chunks, uint32_t span_min)
 {
-    if (DTYPE == OD_BF16) {
-        x[0] = od_bf16_lo(v.x); x[1] = od_bf16_hi(v.x);
-        x[2] = od_bf16_lo(v.y); x[3] = od_bf16_hi(v.y);
-        x[4] = od_bf16_lo(v.z); x[5] = od_bf16_hi(v.z);
-        x[6] = od_bf16_lo(v.w); x[7] = od_bf16_hi(v.w);
-    } else {
-        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
-        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
-    }
+    const uint32_t span = (rows_b * W + n_chunks - 1) / n_chunks;
+    return span < span_min ? span_min : span;
 }
+
+__device__ __forceinline__ int clamp_m(int mb, int K_max) { return mb < 0 ? 0 : (mb > K_max ? K_max : mb); }
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
 {
@@ -82,128 +93,449 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
     return v;
 }
 
-template <int DTYPE>
-__global__ void __launch_bounds__(OD_VERIFY_THREADS)
-od_verify_kernel(const VerifyArgs a)
+// one thread asks the copy engine to pull [p, p + bytes) into L2 (both multiples of 16)
+__device__ __forceinline__ void l2_prefetch_bulk(const void *p, uint32_t bytes)
 {
-    constexpr int VEC = DTYPE == OD_BF16 ? 8 : 4;          // elements per 16 bytes
-    constexpr int UNROLL = 4;
-    const int b = blockIdx.z, r = blockIdx.y, c = blockIdx.x;
-    int mb = a.m[b];
-    mb = mb < 0 ? 0 : (mb > a.K_max ? a.K_max : mb);
-    if (r > mb) return;                                     // rows above m_b are never touched
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 
-    const float T = a.temperature[b];
-    const bool bad_T = !(T > 0.f);
-    const float scale = bad_T ? 0.f : 1.4426950408889634f / T;   // log2(e)/T
-    const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
-    const char *row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)r * a.row_stride) * esz;
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 
-    const int64_t lo = (int64_t)c * a.chunk_elems;
-    int64_t hi = lo + a.chunk_elems;
-    if (hi > a.v_p) hi = a.v_p;
-    const int64_t nvec = (hi - lo) / VEC;                  // whole vectors in this chunk
-    const uint4 *vp = (const uint4 *)(row + (size_t)lo * esz);
+// Packed fp32 pairs (one instruction for two lanes of arithmetic on sm_100).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// acc += (exp2(lo*scale - c), exp2(hi*scale - c))
+__device__ __forceinline__ uint64_t f2_exp_acc(uint64_t acc, float lo, float hi, uint64_t scale2, uint64_t nc2)
+{
+    float e0, e1;
+    f2_unpack(f2_fma(f2_pack(lo, hi), scale2, nc2), e0, e1);
+    return f2_add(acc, f2_pack(od_ex2(e0), od_ex2(e1)));
+}
 
-    float tm = -FLT_MAX, ts = 0.f;
-    int64_t i = threadIdx.x;
-    for (; i + (UNROLL - 1) * OD_VERIFY_THREADS < nvec; i += UNROLL * OD_VERIFY_THREADS) {
-        uint4 v[UNROLL];
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream(vp + i + u * OD_VERIFY_THREADS);
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            float x[8];
-            unpack<DTYPE>(v[u], x);
-            absorb(tm, ts, x, VEC, scale);
-        }
-    }
-    for (; i < nvec; i += OD_VERIFY_THREADS) {
-        float x[8];
-        unpack<DTYPE>(ld_stream(vp + i), x);
-        absorb(tm, ts, x, VEC, scale);
-    }
-    // ragged tail of the row (v_p not a multiple of the vector width)
+// Running state of one thread inside a segment.
+template <int DTYPE>
+struct Lane {
+    float c, s;             // reference exponent (scaled domain), sum of exp2(x*scale - c)
+    float mx;               // fp32 rows: running maximum
+    uint32_t pm;            // bf16 rows: packed running maxima (exact)
+    __device__ __forceinline__ void reset()
     {
-        const int64_t t0 = lo + nvec * VEC + threadIdx.x;
-        if (t0 < hi) {
-            float x[8];
-            x[0] = od_load_logit<DTYPE>(row, t0);
-            absorb(tm, ts, x, 1, scale);
+        c = -FLT_MAX; s = 0.f; mx = -INFINITY; pm = 0xFF80FF80u;
+    }
+    // make c >= gm*scale (branch-free: one rescale per group of vectors)
+    __device__ __forceinline__ void raise(float gm, float scale)
+    {
+        const float cn = fmaxf(fmaxf(gm * scale, -FLT_MAX), c);
+        s *= od_ex2(c - cn);
+        c = cn;
+    }
+    __device__ __forceinline__ float max_seen() const
+    {
+        if (DTYPE == OD_BF16) return fmaxf(od_bf16_lo(pm), od_bf16_hi(pm));
+        return mx;
+    }
+};
+
+// absorb N 16-byte vectors held in registers
+template <int DTYPE, int N>
+__device__ __forceinline__ void absorb(Lane<DTYPE> &L, const uint4 *v, float scale)
+{
+    if (DTYPE == OD_BF16) {
+        uint32_t g = L.pm;
+#pragma unroll
+        for (int u = 0; u < N; ++u) {
+            g = bf16x2_max(g, v[u].x); g = bf16x2_max(g, v[u].y);
+            g = bf16x2_max(g, v[u].z); g = bf16x2_max(g, v[u].w);
+        }
+        L.pm = g;
+        L.raise(fmaxf(od_bf16_lo(g), od_bf16_hi(g)), scale);
+    } else {
+        float gm = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < N; ++u) {
+            gm = fmaxf(gm, fmaxf(fmaxf(__uint_as_float(v[u].x), __uint_as_float(v[u].y)),
+                                 fmaxf(__uint_as_float(v[u].z), __uint_as_float(v[u].w))));
+        }
+        L.mx = fmaxf(L.mx, gm);
+        L.raise(gm, scale);
+    }
+    const uint64_t scale2 = f2_pack(scale, scale), nc2 = f2_pack(-L.c, -L.c);
+    uint64_t a0 = 0ull, a1 = 0ull;                          // two pairs of zeros
+#pragma unroll
+    for (int u = 0; u < N; ++u) {
+        if (DTYPE == OD_BF16) {
+            a0 = f2_exp_acc(a0, od_bf16_lo(v[u].x), od_bf16_hi(v[u].x), scale2, nc2);
+            a1 = f2_exp_acc(a1, od_bf16_lo(v[u].y), od_bf16_hi(v[u].y), scale2, nc2);
+            a0 = f2_exp_acc(a0, od_bf16_lo(v[u].z), od_bf16_hi(v[u].z), scale2, nc2);
+            a1 = f2_exp_acc(a1, od_bf16_lo(v[u].w), od_bf16_hi(v[u].w), scale2, nc2);
+        } else {
+            a0 = f2_exp_acc(a0, __uint_as_float(v[u].x), __uint_as_float(v[u].y), scale2, nc2);
+            a1 = f2_exp_acc(a1, __uint_as_float(v[u].z), __uint_as_float(v[u].w), scale2, nc2);
         }
     }
+    float s0, s1;
+    f2_unpack(f2_add(a0, a1), s0, s1);
+    L.s += s0 + s1;
+}
 
-    // block reduction: shuffle tree inside the warp, then over the warps
+template <int DTYPE>
+__device__ __forceinline__ void absorb_one(Lane<DTYPE> &L, float x, float scale)
+{
+    if (DTYPE == OD_BF16) {
+        // x is a bf16 value: keep the packed maximum exact
+        L.pm = bf16x2_max(L.pm, __float_as_uint(x) >> 16 | 0xFF800000u);
+    } else {
+        L.mx = fmaxf(L.mx, x);
+    }
+    L.raise(x, scale);
+    L.s += od_ex2(fmaf(x, scale, -L.c));
+}
+
+// (c, s) pairs: s counts exp2(x*scale - c)
+__device__ __forceinline__ void pair_merge(float &c, float &s, float c2, float s2)
+{
+    const float cm = fmaxf(c, c2);
+    s = s * od_ex2(c - cm) + s2 * od_ex2(c2 - cm);
+    c = cm;
+}
+
+// all lanes end with the merged (c, s, mx): one rescale per lane, then plain reductions
+__device__ __forceinline__ void warp_merge(float &c, float &s, float &mx)
+{
+    float cm = c;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
-        float m2 = __shfl_xor_sync(0xFFFFFFFFu, tm, off);
-        float s2 = __shfl_xor_sync(0xFFFFFFFFu, ts, off);
-        od_pair_merge(tm, ts, m2, s2, scale);
+        cm = fmaxf(cm, __shfl_xor_sync(0xFFFFFFFFu, cm, off));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
     }
-    __shared__ float sm_m[OD_VERIFY_THREADS / 32], sm_s[OD_VERIFY_THREADS / 32];
-    __shared__ unsigned int s_ticket;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) { sm_m[warp] = tm; sm_s[warp] = ts; }
-    __syncthreads();
+    s *= od_ex2(c - cm);
+    c = cm;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+}
 
-    const int row_slot = b * (a.K_max + 1) + r;
-    if (threadIdx.x == 0) {
-        float bm = sm_m[0], bs = sm_s[0];
-        for (int w = 1; w < OD_VERIFY_THREADS / 32; ++w) od_pair_merge(bm, bs, sm_m[w], sm_s[w], scale);
-        a.partials[(size_t)row_slot * a.chunks + c] = make_float2(bm, bs);
-        __threadfence();
-        s_ticket = atomicAdd(a.row_ticket + row_slot, 1u);
+// Units [v0, v1) of row (b, r) by the whole block; the partial goes to slot `seg` of the row.
+template <int DTYPE>
+__device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r, int seg, int v0, int v1,
+                                              float4 *s_red)
+{
+    constexpr int VEC = DTYPE == OD_BF16 ? 8 : 4;          // elements per 16 bytes
+    constexpr size_t ESZ = DTYPE == OD_BF16 ? 2 : 4;
+    const float T = a.temperature[b];
+    const float scale = (T > 0.f) ? 1.4426950408889634f / T : 0.f;   // log2(e)/T
+    const char *row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)r * a.row_stride) * ESZ;
+    Lane<DTYPE> L;
+    L.reset();
+    // A warp owns whole units (512 bytes, 16 per lane): units v0 + warp, + WARPS, ...
+    // Groups of U units; what is left (1..U-1 units) takes a group of its own
+    // size, so no lane ever computes on padding. Only the row's last unit can be
+    // ragged (lanes past the end of the row, or a final piece under 16 bytes).
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int full_vecs = a.v_p / VEC;                     // whole 16-byte vectors in the row
+    const int full_units = full_vecs >> 5;                 // units whose 32 lanes are all inside
+    const int v1f = v1 < full_units ? v1 : full_units;
+    int v = v0 + warp;
+    const uint4 *p = (const uint4 *)row + (size_t)v * 32 + lane;
+    for (; v + (U - 1) * WARPS < v1f; v += U * WARPS, p += U * WARPS * 32) {
+        uint4 x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) x[u] = ld_stream(p + u * WARPS * 32);
+        absorb<DTYPE, U>(L, x, scale);
     }
+    if (v < v1f) {
+        const int left = (v1f - v + WARPS - 1) / WARPS;    // 1..U-1, the same for the whole warp
+        if (left == 3) {
+            uint4 x[3];
+#pragma unroll
+            for (int u = 0; u < 3; ++u) x[u] = ld_stream(p + u * WARPS * 32);
+            absorb<DTYPE, 3>(L, x, scale);
+        } else if (left == 2) {
+            uint4 x[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) x[u] = ld_stream(p + u * WARPS * 32);
+            absorb<DTYPE, 2>(L, x, scale);
+        } else {
+            uint4 x[1];
+            x[0] = ld_stream(p);
+            absorb<DTYPE, 1>(L, x, scale);
+        }
+    }
+    if (v1 > full_units && warp == ((full_units - v0) & (WARPS - 1))) {
+        // the row's ragged last unit (v1 == W here): whole vectors, then single elements
+        const int i = full_units * 32 + lane;
+        if (i < full_vecs) {
+            uint4 x[1];
+            x[0] = ld_stream((const uint4 *)row + i);
+            absorb<DTYPE, 1>(L, x, scale);
+        }
+        const int e = full_vecs * VEC + lane;
+        if (e < a.v_p) absorb_one<DTYPE>(L, od_load_logit<DTYPE>(row, e), scale);
+    }
+    float c = L.c, s = L.s, mx = L.max_seen();
+    warp_merge(c, s, mx);
+    __syncthreads();                                        // s_red may still be read from the last segment
+    if (lane == 0) s_red[warp] = make_float4(c, s, mx, 0.f);
     __syncthreads();
-    if (s_ticket != (unsigned)(a.chunks - 1)) return;       // not the last block of this row
+    if (warp == 0) {
+        float4 t = lane < WARPS ? s_red[lane] : make_float4(-FLT_MAX, 0.f, -INFINITY, 0.f);
+        c = t.x; s = t.y; mx = t.z;
+        warp_merge(c, s, mx);
+        if (lane == 0)
+            a.partials[((size_t)b * (a.K_max + 1) + r) * OD_VERIFY_SEG_MAX + seg] = make_float4(c, s, mx, 0.f);
+    }
+}
 
-    // ---- last block of the row: merge the chunks in order, decide position r ----
-    if (threadIdx.x != 0) return;
-    __threadfence();
-    a.row_ticket[row_slot] = 0;
-    float M, S;
+template <int DTYPE>
+__global__ void __launch_bounds__(THREADS, OD_VERIFY_BLOCKS_PER_SM)
+od_verify_stream_kernel(const VerifyArgs a)
+{
+    constexpr size_t ESZ = DTYPE == OD_BF16 ? 2 : 4;
+    __shared__ int32_t s_cum[OD_VERIFY_MAX_B + 1];          // exclusive prefix of the clamped m_b
+    __shared__ int32_t s_wsum[WARPS];
+    __shared__ float4 s_red[WARPS];
+
+    // Flat unit indices fit 32 bits (the launcher checks): the walk below is
+    // executed by every thread, so it uses 32-bit arithmetic and as few
+    // divisions as it can (one warp has only a few hundred useful instructions).
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t g = blockIdx.x;
+    const uint32_t W = (uint32_t)a.W;
+
+    // ---- space A (row 0 of every sequence): ask for this block's bytes before anything else
+    const uint32_t a_tot = (uint32_t)a.B * W;
+    uint32_t a_lo = g * (uint32_t)a.span_a;
+    if (a_lo > a_tot) a_lo = a_tot;
+    uint32_t a_hi = a_lo + (uint32_t)a.span_a;
+    if (a_hi > a_tot) a_hi = a_tot;
+    const uint32_t a_b0 = a_lo / W, a_v0 = a_lo - a_b0 * W;   // first sequence and unit of the span
+    if (threadIdx.x == 0 && a_lo < a_hi) {
+        const uint32_t row_bytes16 = (uint32_t)((size_t)a.v_p * ESZ / 16 * 16);
+        uint32_t f = a_lo, b = a_b0, v0 = a_v0;
+        while (f < a_hi) {
+            uint32_t n = a_hi - f;
+            if (n > W - v0) n = W - v0;
+            const char *row = (const char *)a.logits + (size_t)b * a.seq_stride * ESZ;
+            uint32_t lo = v0 * 512u, hi = (v0 + n) * 512u;
+            if (hi > row_bytes16) hi = row_bytes16;
+            if (hi > lo) l2_prefetch_bulk(row + lo, hi - lo);
+            f += n; ++b; v0 = 0;
+        }
+    }
+
+    // everything below may read what the translation kernel wrote
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+
+    // ---- prefix sums of m (clamped) for space B
     {
-        const volatile float2 *pp = (const volatile float2 *)(a.partials + (size_t)row_slot * a.chunks);
-        M = pp[0].x; S = pp[0].y;
-        for (int k = 1; k < a.chunks; ++k) od_pair_merge(M, S, pp[k].x, pp[k].y, scale);
+        const int per = (a.B + THREADS - 1) / THREADS;
+        const int i0 = threadIdx.x * per;
+        int loc = 0;
+        for (int i = i0; i < i0 + per && i < a.B; ++i) loc += clamp_m(a.m[i], a.K_max);
+        int inc = loc;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+            if (lane >= off) inc += t;
+        }
+        if (lane == 31) s_wsum[warp] = inc;
+        __syncthreads();
+        int base = 0;
+        for (int w = 0; w < warp; ++w) base += s_wsum[w];
+        int run = base + inc - loc;
+        for (int i = i0; i < i0 + per && i < a.B; ++i) {
+            s_cum[i] = run;
+            run += clamp_m(a.m[i], a.K_max);
+        }
+        if (threadIdx.x == THREADS - 1) s_cum[a.B] = base + inc;
+        __syncthreads();
     }
-    a.row_max[row_slot] = M;
-    a.row_sum[row_slot] = S;
-    unsigned int bits = 0;
-    if (!(S > 0.f) || !(S <= FLT_MAX)) atomicOr(a.seq_bits + 2 * b + 1, 1u);   // not finite and positive
-    if (r < mb) {
+
+    // ---- space A: a row that starts inside this span has its segment 0 here
+    if (a_lo < a_hi) {
+        uint32_t f = a_lo, b = a_b0, v0 = a_v0;
+        uint32_t seg = g - (a_lo - a_v0) / (uint32_t)a.span_a;
+        while (f < a_hi) {
+            uint32_t n = a_hi - f;
+            if (n > W - v0) n = W - v0;
+            block_segment<DTYPE>(a, (int)b, 0, (int)seg, (int)v0, (int)(v0 + n), s_red);
+            f += n; ++b; v0 = 0; seg = 0;
+        }
+    }
+
+    // ---- space B (rows 1..m_b), spans handed out from the other end of the grid
+    {
+        const uint32_t rows_b = (uint32_t)s_cum[a.B];
+        const uint32_t b_tot = rows_b * W;
+        if (b_tot == 0) return;
+        uint32_t span = (b_tot + (uint32_t)a.n_chunks - 1) / (uint32_t)a.n_chunks;
+        if (span < (uint32_t)a.span_min) span = (uint32_t)a.span_min;
+        const uint32_t chunk = (uint32_t)a.n_chunks - 1 - g;
+        uint32_t f = chunk * span;
+        if (f >= b_tot) return;
+        uint32_t f_hi = f + span;
+        if (f_hi > b_tot) f_hi = b_tot;
+        uint32_t rho = f / W, v0 = f - rho * W;
+        uint32_t seg = chunk - (f - v0) / span;
+        // sequence holding flat row rho: the last b with cum[b] <= rho (skips m_b = 0)
+        int lo = 0, hi = a.B;                                // invariant: cum[lo] <= rho < cum[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if ((uint32_t)s_cum[mid] <= rho) lo = mid; else hi = mid;
+        }
+        int b = lo;
+        while (f < f_hi) {
+            while ((uint32_t)s_cum[b + 1] <= rho) ++b;
+            uint32_t n = f_hi - f;
+            if (n > W - v0) n = W - v0;
+            block_segment<DTYPE>(a, b, 1 + (int)(rho - (uint32_t)s_cum[b]), (int)seg, (int)v0, (int)(v0 + n), s_red);
+            f += n; ++rho; v0 = 0; seg = 0;
+        }
+    }
+}
+
+// One block per sequence, warp r = row r (blockDim = 32 * (K_max + 1)).
+template <int DTYPE>
+__global__ void __launch_bounds__(32 * (OD_MAX_K + 1))
+od_verify_decide_kernel(const VerifyArgs a)
+{
+    constexpr size_t ESZ = DTYPE == OD_BF16 ? 2 : 4;
+    __shared__ int32_t s_part[2][OD_MAX_K + 1];
+    __shared__ unsigned int s_bits[2];
+
+    const int b = blockIdx.x;
+    const int lane = threadIdx.x & 31, r = threadIdx.x >> 5;
+    const uint32_t W = (uint32_t)a.W;
+
+    // ---- before the stream kernel has finished: everything that does not depend on it.
+    // (m, the target ids and q' come from the translation kernel, which was complete
+    // before any block of the stream kernel let this grid start.)
+    int before = 0, total = 0;                               // sums of clamped m over [0, b) and [0, B)
+    for (int i = threadIdx.x; i < a.B; i += blockDim.x) {
+        const int v = clamp_m(a.m[i], a.K_max);
+        total += v;
+        if (i < b) before += v;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        before += __shfl_xor_sync(0xFFFFFFFFu, before, off);
+        total += __shfl_xor_sync(0xFFFFFFFFu, total, off);
+    }
+    if (lane == 0) { s_part[0][r] = before; s_part[1][r] = total; }
+    if (threadIdx.x == 0) { s_bits[0] = 0; s_bits[1] = 0; }
+    const int mb = clamp_m(a.m[b], a.K_max);
+    const float T = a.temperature[b];
+    const bool bad_T = !(T > 0.f);
+    const float scale = bad_T ? 0.f : 1.4426950408889634f / T;
+    const char *row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)r * a.row_stride) * ESZ;
+    float x_t = 0.f, q = 0.f, u = 0.f;
+    bool t_ok = false;
+    if (lane == 0 && r < mb) {
         const size_t o = (size_t)b * a.K_max + r;
         const int32_t t = a.tgt_ids[o];
-        float p = 0.f;
-        if (t >= 0 && t < a.v_p) p = od_ex2((od_load_logit<DTYPE>(row, t) - M) * scale) / S;
-        const float q = a.q_prime[o];
-        const float ra = (q <= p) ? 1.f : p / q;
-        const float u = od_uniform(a.seed[b], a.step, (uint32_t)r, 0u);
-        a.p_sel[o] = p;
-        a.ratio[o] = ra;
-        if (u < ra) bits |= 1u << r;
-        if (fabsf(u - ra) <= OD_TAU_ACCEPT) bits |= 1u << (16 + r);
+        t_ok = t >= 0 && t < a.v_p;
+        if (t_ok) x_t = od_load_logit<DTYPE>(row, t);
+        q = a.q_prime[o];
+        u = od_uniform(a.seed[b], a.step, (uint32_t)r, 0u);
     }
-    if (bits) atomicOr(a.seq_bits + 2 * b, bits);
-    __threadfence();
-    const unsigned int st = atomicAdd(a.seq_ticket + b, 1u);
-    if (st != (unsigned)mb) return;                         // rows 0..m_b: m_b + 1 tickets
+    __syncthreads();
+    before = 0; total = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { before += s_part[0][w]; total += s_part[1][w]; }
 
-    // ---- last row of the sequence: accepted prefix ----
-    __threadfence();
-    const unsigned int all = atomicExch(a.seq_bits + 2 * b, 0u);
-    const unsigned int misc = atomicExch(a.seq_bits + 2 * b + 1, 0u);
-    a.seq_ticket[b] = 0;
-    int n = 0;
-    while (n < mb && (all >> n & 1u)) ++n;
-    int nd = 0;
-    for (int k = 0; k < n; ++k) nd += a.span_len[(size_t)b * a.K_max + k];
-    uint32_t f = (all >> 16) & OD_VF_BOUNDARY_MASK;
-    if (misc & 1u) f |= OD_VF_NONFINITE;
-    if (bad_T) { f |= OD_VF_BAD_TEMPERATURE; n = 0; nd = 0; }
-    a.n_accepted[b] = n;
-    a.n_draft_accepted[b] = nd;
-    a.flags[b] = f;
+    int nseg = 0;
+    if (r <= mb) {
+        if (r == 0) nseg = row_segments((uint32_t)b, W, (uint32_t)a.span_a);
+        else nseg = row_segments((uint32_t)(before + r - 1), W,
+                                 span_of_space_b((uint32_t)total, W, (uint32_t)a.n_chunks, (uint32_t)a.span_min));
+    }
+
+    // ---- the partials
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+
+    if (r <= mb) {
+        const int row_slot = b * (a.K_max + 1) + r;
+        const float4 *pp = a.partials + (size_t)row_slot * OD_VERIFY_SEG_MAX;
+        float c = -FLT_MAX, s = 0.f, mx = -INFINITY;
+        for (int k = lane; k < nseg; k += 32) {
+            const float4 p = __ldcg(pp + k);
+            pair_merge(c, s, p.x, p.y);
+            mx = fmaxf(mx, p.z);
+        }
+        warp_merge(c, s, mx);
+        if (lane == 0) {
+            const float M = mx;
+            const float S = s * od_ex2(fmaf(-M, scale, c));     // sum of exp2((x - M)*scale)
+            a.row_max[row_slot] = M;
+            a.row_sum[row_slot] = S;
+            if (!(S > 0.f) || !(S <= FLT_MAX)) atomicOr(&s_bits[1], 1u);   // not finite and positive
+            if (r < mb) {
+                const size_t o = (size_t)b * a.K_max + r;
+                const float p = t_ok ? od_ex2((x_t - M) * scale) / S : 0.f;
+                const float ra = (q <= p) ? 1.f : p / q;
+                a.p_sel[o] = p;
+                a.ratio[o] = ra;
+                unsigned int bits = 0;
+                if (u < ra) bits |= 1u << r;
+                if (fabsf(u - ra) <= OD_TAU_ACCEPT) bits |= 1u << (16 + r);
+                if (bits) atomicOr(&s_bits[0], bits);
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int all = s_bits[0];
+        int n = 0;
+        while (n < mb && (all >> n & 1u)) ++n;
+        int nd = 0;
+        for (int k = 0; k < n; ++k) nd += a.span_len[(size_t)b * a.K_max + k];
+        uint32_t f = (all >> 16) & OD_VF_BOUNDARY_MASK;
+        if (s_bits[1] & 1u) f |= OD_VF_NONFINITE;
+        if (bad_T) { f |= OD_VF_BAD_TEMPERATURE; n = 0; nd = 0; }
+        a.n_accepted[b] = n;
+        a.n_draft_accepted[b] = nd;
+        a.flags[b] = f;
+    }
+}
+
+template <typename Kern>
+cudaError_t launch(Kern kern, unsigned grid, unsigned block, cudaStream_t s, bool pdl, const VerifyArgs &a)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
 }  // namespace
@@ -217,44 +549,54 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              int32_t *n_accepted, int32_t *n_draft_accepted,
                              uint32_t *flags, cudaStream_t s)
 {
-    if (B == 0) return cudaSuccess;
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
     const int64_t row_bytes = (int64_t)c->v_p * esz;
-    const int64_t gran = 4096;                              // 256 threads x 16 bytes
-    int64_t chunk_bytes = c->opt_verify_chunk_bytes;
-    if (chunk_bytes <= 0) {
-        // enough blocks to fill the machine several times over, chunks of 8..64 KB
-        const int64_t rows = (int64_t)B * (K_max + 1);
-        const int64_t want_blocks = (int64_t)c->sm_count * 16;
-        int64_t per_row = (want_blocks + rows - 1) / rows;
-        if (per_row < 1) per_row = 1;
-        chunk_bytes = (row_bytes + per_row - 1) / per_row;
-        if (chunk_bytes < 8192) chunk_bytes = 8192;
-        if (chunk_bytes > 65536) chunk_bytes = 65536;
+    const int32_t W = (int32_t)((row_bytes + 511) / 512);
+    const int32_t span_min = (W + OD_VERIFY_SEG_MAX - 2) / (OD_VERIFY_SEG_MAX - 1);
+    int64_t blocks_per_sm = c->opt_verify_blocks_per_sm > 0 ? c->opt_verify_blocks_per_sm : OD_VERIFY_BLOCKS_PER_SM;
+    if (blocks_per_sm > OD_VERIFY_BLOCKS_PER_SM) blocks_per_sm = OD_VERIFY_BLOCKS_PER_SM;
+
+    // batches beyond the shared-memory prefix table go in slices; a slice's flat
+    // unit indices (plus one span of slack) must fit 32 bits
+    int32_t slice = OD_VERIFY_MAX_B;
+    while (slice > 1 && (int64_t)slice * (K_max + 1) * W > (int64_t)1 << 30) slice >>= 1;
+    for (int32_t b0 = 0; b0 < B; b0 += slice) {
+        const int32_t nb = B - b0 < slice ? B - b0 : slice;
+        // no more blocks than the most this slice can need
+        const int64_t max_units = (int64_t)nb * (K_max + 1) * W;
+        int64_t grid = (int64_t)c->sm_count * blocks_per_sm;
+        const int64_t need = max_units / span_min + 1;
+        if (grid > need) grid = need;
+        if (grid < 1) grid = 1;
+        VerifyArgs a;
+        a.logits = (const char *)logits + (size_t)b0 * seq_stride * esz;
+        a.row_stride = row_stride; a.seq_stride = seq_stride;
+        a.B = nb; a.K_max = K_max; a.v_p = c->v_p;
+        a.W = W; a.n_chunks = (int32_t)grid; a.span_min = span_min;
+        int64_t span_a = ((int64_t)nb * W + grid - 1) / grid;
+        if (span_a < span_min) span_a = span_min;
+        a.span_a = (int32_t)span_a;
+        a.tgt_ids = tgt_ids + (size_t)b0 * K_max; a.q_prime = q_prime + (size_t)b0 * K_max;
+        a.span_len = span_len + (size_t)b0 * K_max; a.m = m + b0;
+        a.temperature = temperature + b0; a.seed = seed + b0; a.step = step;
+        a.row_max = row_max + (size_t)b0 * (K_max + 1); a.row_sum = row_sum + (size_t)b0 * (K_max + 1);
+        a.p_sel = p_sel + (size_t)b0 * K_max; a.ratio = ratio + (size_t)b0 * K_max;
+        a.n_accepted = n_accepted + b0; a.n_draft_accepted = n_draft_accepted + b0;
+        a.flags = flags + b0;
+        a.partials = c->d_partials;
+        c->info[0] = grid;
+        c->info[1] = span_a;
+
+        const bool pdl = c->opt_pdl != 0;
+        cudaError_t e = dtype == OD_BF16
+            ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)grid, THREADS, s, pdl, a)
+            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)grid, THREADS, s, pdl, a);
+        if (e != cudaSuccess) return e;
+        const unsigned dthreads = 32u * (unsigned)(K_max + 1);
+        e = dtype == OD_BF16
+            ? launch(od_verify_decide_kernel<OD_BF16>, (unsigned)nb, dthreads, s, pdl, a)
+            : launch(od_verify_decide_kernel<OD_F32>, (unsigned)nb, dthreads, s, pdl, a);
+        if (e != cudaSuccess) return e;
     }
-    chunk_bytes = (chunk_bytes + gran - 1) / gran * gran;
-    int64_t chunks = (row_bytes + chunk_bytes - 1) / chunk_bytes;
-    if (chunks > c->max_chunks) {                           // scratch was sized for 4 KB chunks at most
-        chunks = c->max_chunks;
-        chunk_bytes = ((row_bytes + chunks - 1) / chunks + gran - 1) / gran * gran;
-        chunks = (row_bytes + chunk_bytes - 1) / chunk_bytes;
-    }
-    VerifyArgs a;
-    a.logits = logits; a.row_stride = row_stride; a.seq_stride = seq_stride;
-    a.B = B; a.K_max = K_max; a.v_p = c->v_p;
-    a.chunk_elems = (int32_t)(chunk_bytes / esz); a.chunks = (int32_t)chunks;
-    a.tgt_ids = tgt_ids; a.q_prime = q_prime; a.span_len = span_len; a.m = m;
-    a.temperature = temperature; a.seed = seed; a.step = step;
-    a.row_max = row_max; a.row_sum = row_sum; a.p_sel = p_sel; a.ratio = ratio;
-    a.n_accepted = n_accepted; a.n_draft_accepted = n_draft_accepted; a.flags = flags;
-    a.partials = c->d_partials; a.row_ticket = c->d_row_ticket;
-    a.seq_ticket = c->d_seq_ticket; a.seq_bits = c->d_seq_bits;
-    dim3 grid((unsigned)chunks, (unsigned)(K_max + 1), (unsigned)B);
-    c->info[0] = (int64_t)chunks * (K_max + 1) * B;
-    c->info[1] = a.chunk_elems;
-    if (dtype == OD_BF16)
-        od_verify_kernel<OD_BF16><<<grid, OD_VERIFY_THREADS, 0, s>>>(a);
-    else
-        od_verify_kernel<OD_F32><<<grid, OD_VERIFY_THREADS, 0, s>>>(a);
-    return cudaGetLastError();
+    return cudaSuccess;
 }

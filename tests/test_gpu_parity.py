@@ -78,11 +78,11 @@ def test_cache_hits_and_unmapped_stops_are_exercised(cuda_device):
     assert s.cache_hits > 50 and s.unmapped_stops > 5
 
 
-@pytest.mark.parametrize("chunk_bytes,tiles", [(4096, 1), (8192, 2), (65536, 7), (1 << 20, 1000)])
-def test_every_split_of_a_row_gives_the_same_answer(cuda_device, chunk_bytes, tiles):
+@pytest.mark.parametrize("blocks_per_sm,tiles,pdl", [(1, 1, 1), (2, 2, 0), (4, 7, 1), (8, 1000, 0)])
+def test_every_split_of_a_row_gives_the_same_answer(cuda_device, blocks_per_sm, tiles, pdl):
     w = _small("split", v_q=3000, v_p=20011, B=5, cache_entries=500, gen_seed=0xBEEF40)
     _run_workload(w, cuda_device, range(3), pad=True,
-                  opts={"verify_chunk_bytes": chunk_bytes, "sample_tiles_per_block": tiles})
+                  opts={"verify_blocks_per_sm": blocks_per_sm, "sample_tiles_per_warp": tiles, "pdl": pdl})
 
 
 def test_max_k_and_zero_length_proposals(cuda_device):
