@@ -57,7 +57,8 @@ enum od_status {
     OD_ERR_UNSUPPORTED = -5,       /* dtype, vocabulary too large for the cache key */
     OD_ERR_CUDA = -6,              /* a CUDA runtime call failed */
     OD_ERR_NOMEM = -7,
-    OD_ERR_STATE = -8              /* call out of order (e.g. no vocabulary map yet) */
+    OD_ERR_STATE = -8,             /* call out of order (e.g. no vocabulary map yet) */
+    OD_ERR_SCRATCH_LIMIT = -9      /* od_verify_noalloc: batch too large for its fixed scratch */
 };
 
 enum od_dtype { OD_F32 = 0, OD_BF16 = 1 };
@@ -96,6 +97,7 @@ enum od_counter {
 #define OD_TAU_SAMPLE 2.0e-6
 
 #define OD_MAX_K 16      /* largest K_max */
+#define OD_NOALLOC_MAX_ROWS 1024 /* od_verify_noalloc: largest B * (K_max + 1) */
 #define OD_NGRAM_MAX 4   /* longest cached run */
 
 /* ---- context ----------------------------------------------------------- */
@@ -218,6 +220,50 @@ int32_t od_sample_residual(od_ctx *ctx, int32_t B, int32_t K_max,
                            const uint64_t *seed, uint64_t step,
                            int32_t *out_token, float *resid_mass,
                            uint32_t *sample_flags, void *stream);
+
+/* Step 2 without any allocation (the paper has no counterpart: this entry
+ * point exists for the way some programs are built, not for the method).
+ *
+ * Who needs it: a caller that is handed its buffers and must not ask the CUDA
+ * runtime for device memory itself. Typical cases are a plug-in inside a
+ * serving process whose own allocator reserved the GPU's memory at start-up,
+ * so a cudaMalloc from a library would fail or eat into memory the host
+ * application budgeted, and a decode loop that cannot afford the device-wide
+ * synchronisation cudaMalloc and cudaFree imply. Such a caller cannot use
+ * od_create (which allocates the maps, the cache table and the kernels'
+ * scratch), so this function takes no context: the target vocabulary size is an
+ * argument, and it works on the CUDA device that is current when it is called.
+ *
+ * What it computes: exactly od_verify (same kernels, same arithmetic, same
+ * outputs and flags; see above for the arguments, all device pointers owned by
+ * the caller). What differs is the kernels' scratch, the per-segment partial
+ * sums of the streaming pass: it is a fixed 1 MiB array compiled into the
+ * library (OD_NOALLOC_MAX_ROWS rows x 64 partials x 16 bytes) that every GPU
+ * loading the library holds until the process ends. The function calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Limits and rules
+ *   - B * (K_max + 1) <= OD_NOALLOC_MAX_ROWS and B <= 2048; anything larger is
+ *     refused with OD_ERR_SCRATCH_LIMIT before any launch.
+ *   - The first call on a device looks up the array's device address and the
+ *     multiprocessor count (no allocation, but host-side runtime calls): make
+ *     that first call during start-up, before any stream capture begins.
+ *   - All calls on a device share the one array. It keeps whatever the last
+ *     call left in it; nothing in it needs clearing, because a call reads only
+ *     the slots it has written itself. Two calls whose kernels overlap on the
+ *     GPU (different streams, no dependency between them) race on it: order
+ *     them. Calls on one stream are ordered.
+ *   - Asynchronous on `stream` like od_verify; errors as for od_verify. */
+int32_t od_verify_noalloc(int32_t target_vocab, int32_t B, int32_t K_max,
+                          const void *logits, int32_t logit_dtype,
+                          int64_t row_stride, int64_t seq_stride,
+                          const int32_t *tgt_ids, const float *q_prime,
+                          const int32_t *span_len, const int32_t *m,
+                          const float *temperature, const uint64_t *seed,
+                          uint64_t step, float *row_max, float *row_sum,
+                          float *p_sel, float *ratio, int32_t *n_accepted,
+                          int32_t *n_draft_accepted, uint32_t *verify_flags,
+                          void *stream);
 
 /* ---- whole step from host memory ---------------------------------------- */
 

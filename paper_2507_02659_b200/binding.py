@@ -26,10 +26,11 @@ OD_VF_BOUNDARY_MASK, OD_VF_BAD_TEMPERATURE, OD_VF_NONFINITE = 0xFFFF, 0x10000, 0
 OD_SF_BOUNDARY, OD_SF_ZERO_MASS, OD_SF_BAD_TEMPERATURE, OD_SF_BONUS = 0x1, 0x2, 0x4, 0x10
 OD_TAU_ACCEPT, OD_TAU_SAMPLE = 1.0e-5, 2.0e-6
 OD_MAX_K = 16
+OD_NOALLOC_MAX_ROWS = 1024
 
 EXPORTS = ["od_create", "od_destroy", "od_set_vocab_map", "od_cache_build", "od_set_option",
            "od_map_proposals", "od_verify", "od_sample_residual", "od_host_step_reserve",
-           "od_step_host", "od_last_launch_info", "od_status_string", "od_version"]
+           "od_step_host", "od_verify_noalloc", "od_last_launch_info", "od_status_string", "od_version"]
 
 
 class OdError(RuntimeError):
@@ -61,6 +62,7 @@ def lib():
         L.od_verify.argtypes = [vp, i32, i32, vp, i32, i64, i64] + [vp] * 6 + [u64] + [vp] * 7 + [vp]
         L.od_sample_residual.argtypes = ([vp, i32, i32, vp, i32, i64, i64] + [vp] * 13 + [u64]
                                          + [vp] * 3 + [vp])
+        L.od_verify_noalloc.argtypes = [i32, i32, i32, vp, i32, i64, i64] + [vp] * 6 + [u64] + [vp] * 7 + [vp]
         L.od_host_step_reserve.argtypes = [vp, i32]
         L.od_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp, u64] + [vp] * 7 + [vp]
         L.od_last_launch_info.argtypes = [vp, i32]
@@ -245,6 +247,27 @@ def od_verify(ctx: Context, logits, mp: MapOut, temperature, seed, step: int,
         _dp(out.row_max, f32, d), _dp(out.row_sum, f32, d), _dp(out.p_sel, f32, d),
         _dp(out.ratio, f32, d), _dp(out.n_accepted, i32, d), _dp(out.n_draft_accepted, i32, d),
         _dp(out.flags, i32, d), _stream(d)), "od_verify")
+    return out
+
+
+def od_verify_noalloc(target_vocab: int, logits, mp: MapOut, temperature, seed, step: int,
+                      out: VerifyOut) -> VerifyOut:
+    """od_verify for callers that may not allocate device memory: no context, the
+    kernels' scratch is a fixed array inside the library, and `out` must be passed
+    in (this wrapper allocates nothing either). Works on the device of `logits`,
+    which must be the current CUDA device."""
+    B, K = mp.tgt_ids.shape
+    d, i32, f32 = logits.device, torch.int32, torch.float32
+    if d.type != "cuda" or d.index != torch.cuda.current_device():
+        raise ValueError("logits must live on the current CUDA device")
+    rs, ss = _strides(logits, B, K, target_vocab)
+    _check(lib().od_verify_noalloc(
+        target_vocab, B, K, C.c_void_p(logits.data_ptr()), logit_dtype_code(logits), rs, ss,
+        _dp(mp.tgt_ids, i32, d), _dp(mp.q_prime, f32, d), _dp(mp.span_len, i32, d), _dp(mp.m, i32, d),
+        _dp(temperature, f32, d), _dp(seed, torch.int64, d), C.c_uint64(step & (2**64 - 1)),
+        _dp(out.row_max, f32, d), _dp(out.row_sum, f32, d), _dp(out.p_sel, f32, d),
+        _dp(out.ratio, f32, d), _dp(out.n_accepted, i32, d), _dp(out.n_draft_accepted, i32, d),
+        _dp(out.flags, i32, d), _stream(d)), "od_verify_noalloc")
     return out
 
 

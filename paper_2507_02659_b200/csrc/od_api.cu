@@ -401,6 +401,7 @@ const char *od_status_string(int32_t status)
         case OD_ERR_CUDA: return "CUDA runtime error";
         case OD_ERR_NOMEM: return "out of memory";
         case OD_ERR_STATE: return "call out of order";
+        case OD_ERR_SCRATCH_LIMIT: return "batch too large for the fixed scratch of od_verify_noalloc";
         default: return "unknown status";
     }
 }
