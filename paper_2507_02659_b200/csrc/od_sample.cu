@@ -51,31 +51,30 @@ struct SampleArgs {
 struct SeqState {
     const char *row;
     const float *q_row;
-    float M, invS, scale;
+    float M, S, scale;
     bool residual;
     int32_t ngram_token, prefix_token;
     float ngram_prob, prefix_val;
 };
 
-__device__ __forceinline__ float r_of(const SeqState &q, bool residual, int64_t t, float x, int32_t d)
+// Values are carried UNNORMALISED: with e(t) = exp2((x_t - M)*scale) = p(t)*S,
+//   residual   r'(t) = max(0, e(t) - q'(t)*S) = S * max(0, p(t) - q'(t))
+//   free token r'(t) = e(t)
+// so one multiplication by 1/S at the very end replaces one per element, and the
+// inverse-CDF pick (target = u * sum r') is unchanged by the common factor.
+__device__ __forceinline__ float resid_of(const SeqState &q, float x, float qq)
 {
-    const float p = od_ex2((x - q.M) * q.scale) * q.invS;
-    if (!residual) return p;
-    float qq = d >= 0 ? __ldg(q.q_row + d) : 0.f;
-    if (t == q.prefix_token) qq = q.prefix_val;
-    if (t == q.ngram_token) qq = q.ngram_prob;
-    return fmaxf(0.f, p - qq);
+    return fmaxf(0.f, fmaf(-qq, q.S, od_ex2((x - q.M) * q.scale)));
 }
 
-// r(t) of the EPT consecutive ids this lane owns in `tile`; ids >= v_p give 0
+// r'(t) of the EPT consecutive ids this lane owns in `tile`; ids >= v_p give 0
 template <int DTYPE>
 __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs &a, bool residual,
                                             int tile, int lane, float *r)
 {
-    const int64_t t0 = (int64_t)tile * OD_SAMPLE_TILE + (int64_t)lane * EPT;
+    const int t0 = tile * OD_SAMPLE_TILE + lane * EPT;
     if (t0 + EPT <= a.v_p) {
         float x[EPT];
-        int32_t d[EPT];
         if (DTYPE == OD_BF16) {
             const uint4 v = __ldg((const uint4 *)(q.row + (size_t)t0 * 2));
             x[0] = od_bf16_lo(v.x); x[1] = od_bf16_hi(v.x); x[2] = od_bf16_lo(v.y); x[3] = od_bf16_hi(v.y);
@@ -89,32 +88,57 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
         if (residual) {
             const int4 i0 = __ldg((const int4 *)(a.inv_map + t0));
             const int4 i1 = __ldg((const int4 *)(a.inv_map + t0) + 1);
-            d[0] = i0.x; d[1] = i0.y; d[2] = i0.z; d[3] = i0.w;
-            d[4] = i1.x; d[5] = i1.y; d[6] = i1.z; d[7] = i1.w;
-        }
+            const int32_t d[EPT] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
+            float qq[EPT];
 #pragma unroll
-        for (int e = 0; e < EPT; ++e) r[e] = r_of(q, residual, t0 + e, x[e], residual ? d[e] : -1);
+            for (int e = 0; e < EPT; ++e) qq[e] = d[e] >= 0 ? __ldg(q.q_row + d[e]) : 0.f;
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) r[e] = resid_of(q, x[e], qq[e]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) r[e] = od_ex2((x[e] - q.M) * q.scale);
+        }
     } else {
 #pragma unroll
         for (int e = 0; e < EPT; ++e) {
-            const int64_t t = t0 + e;
+            const int t = t0 + e;
+            r[e] = 0.f;
             if (t < a.v_p) {
                 const float xv = od_load_logit<DTYPE>(q.row, t);
-                const int32_t dv = residual ? __ldg(a.inv_map + t) : -1;
-                r[e] = r_of(q, residual, t, xv, dv);
-            } else {
-                r[e] = 0.f;
+                if (residual) {
+                    const int32_t dv = __ldg(a.inv_map + t);
+                    r[e] = resid_of(q, xv, dv >= 0 ? __ldg(q.q_row + dv) : 0.f);
+                } else {
+                    r[e] = od_ex2((xv - q.M) * q.scale);
+                }
             }
+        }
+    }
+    if (residual) {
+        // Eq. (2): the two ids whose q' is not the drafter's row. Only the lane that
+        // owns such an id redoes it (prefix sub-token first, the n-gram token last).
+        const int dp = q.prefix_token - t0, dn = q.ngram_token - t0;
+        if ((unsigned)dp < (unsigned)EPT && q.prefix_token < a.v_p) {
+            const float v = resid_of(q, od_load_logit<DTYPE>(q.row, q.prefix_token), q.prefix_val);
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) r[e] = e == dp ? v : r[e];
+        }
+        if ((unsigned)dn < (unsigned)EPT && q.ngram_token < a.v_p) {
+            const float v = resid_of(q, od_load_logit<DTYPE>(q.row, q.ngram_token), q.ngram_prob);
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) r[e] = e == dn ? v : r[e];
         }
     }
 }
 
+// a lane's eight values are added in fp32 in index order (both passes do exactly
+// this); everything across lanes and tiles is fp64
 __device__ __forceinline__ double lane_sum(const float *r)
 {
-    double s = 0.0;
+    float s = r[0];
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) s += (double)r[e];
-    return s;
+    for (int e = 1; e < EPT; ++e) s += r[e];
+    return (double)s;
 }
 
 __device__ __forceinline__ double warp_sum(double v)
@@ -179,7 +203,7 @@ od_sample_kernel(const SampleArgs a)
     SeqState q;
     q.row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)j * a.row_stride) * esz;
     q.M = a.row_max[b * (K + 1) + j];
-    q.invS = 1.f / a.row_sum[b * (K + 1) + j];
+    q.S = a.row_sum[b * (K + 1) + j];
     q.scale = 1.4426950408889634f / T;
     q.residual = (j < mb) || stop;
     q.ngram_token = -1; q.prefix_token = -1; q.ngram_prob = 0.f; q.prefix_val = 0.f;
@@ -287,7 +311,8 @@ od_sample_kernel(const SampleArgs a)
     }
     if (s_tile < 0 || s_tile == 0x7FFFFFFF) {       // no mass at all (non-finite input)
         if (threadIdx.x == 0) {
-            a.out_token[b] = -1; a.resid_mass[b] = (float)s_total; a.flags[b] = flags | OD_SF_ZERO_MASS;
+            a.out_token[b] = -1; a.resid_mass[b] = (float)(s_total / (double)q.S);
+            a.flags[b] = flags | OD_SF_ZERO_MASS;
             a.ticket[b] = 0;
         }
         return;
@@ -296,7 +321,7 @@ od_sample_kernel(const SampleArgs a)
 
     // ---- warp 0 scans inside the chosen tile ----
     const int tile = s_tile;
-    const double R = s_total;
+    const double Rn = s_total;                      // unnormalised total
     float r[EPT];
     tile_values<DTYPE>(q, a, residual, tile, lane, r);
     const double mine = lane_sum(r);
@@ -306,15 +331,18 @@ od_sample_kernel(const SampleArgs a)
         const double v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
         if (lane >= off) incl += v;
     }
-    double c = s_before + (incl - mine);
-    const int64_t t0 = (int64_t)tile * OD_SAMPLE_TILE + (int64_t)lane * EPT;
+    const double base = s_before + (incl - mine);   // sum before this lane's first id
+    const int t0 = tile * OD_SAMPLE_TILE + lane * EPT;
     int my_pick = 0x7FFFFFFF, my_last = -1;
     double lo = 0.0, hi = 0.0;
+    float run = 0.f;                                // same fp32 order as lane_sum
+    double c = base;
 #pragma unroll
     for (int e = 0; e < EPT; ++e) {
-        const double nc = c + (double)r[e];
-        if (r[e] > 0.f) my_last = (int)(t0 + e);
-        if (my_pick == 0x7FFFFFFF && nc > target) { my_pick = (int)(t0 + e); lo = c; hi = nc; }
+        run = e == 0 ? r[0] : run + r[e];
+        const double nc = base + (double)run;
+        if (r[e] > 0.f) my_last = t0 + e;
+        if (my_pick == 0x7FFFFFFF && nc > target) { my_pick = t0 + e; lo = c; hi = nc; }
         c = nc;
     }
     int pick = my_pick, last = my_last;
@@ -323,19 +351,20 @@ od_sample_kernel(const SampleArgs a)
         pick = min(pick, __shfl_xor_sync(0xFFFFFFFFu, pick, off));
         last = max(last, __shfl_xor_sync(0xFFFFFFFFu, last, off));
     }
+    const float R = (float)(Rn / (double)q.S);      // residual mass (1 for the free token)
     if (pick != 0x7FFFFFFF) {
         if (my_pick == pick) {                      // exactly one lane owns the picked id
             const double margin = fmin(target - lo, hi - target);
-            if (margin <= OD_TAU_SAMPLE * R) flags |= OD_SF_BOUNDARY;
+            if (margin <= OD_TAU_SAMPLE * Rn) flags |= OD_SF_BOUNDARY;
             a.out_token[b] = pick;
-            a.resid_mass[b] = (float)R;
+            a.resid_mass[b] = R;
             a.flags[b] = flags;
             a.ticket[b] = 0;
         }
     } else if (lane == 0) {
         // rounding: target beyond the tile's last edge
         a.out_token[b] = last;
-        a.resid_mass[b] = (float)R;
+        a.resid_mass[b] = R;
         a.flags[b] = flags | OD_SF_BOUNDARY | (last < 0 ? OD_SF_ZERO_MASS : 0u);
         a.ticket[b] = 0;
     }
