@@ -58,6 +58,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--verify-blocks-per-sm", type=int, default=0)
+    ap.add_argument("--verify-waves", type=int, default=0)
     ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches")
     return ap.parse_args()
@@ -236,6 +237,8 @@ def main():
     ctx.cache_build(st.runs, st.run_len, st.run_target)
     if a.verify_blocks_per_sm:
         ctx.set_option("verify_blocks_per_sm", a.verify_blocks_per_sm)
+    if a.verify_waves:
+        ctx.set_option("verify_waves", a.verify_waves)
     if a.sample_tiles_per_warp:
         ctx.set_option("sample_tiles_per_warp", a.sample_tiles_per_warp)
     if a.no_pdl:

@@ -40,6 +40,7 @@ struct od_ctx {
 
     // options
     int64_t opt_verify_blocks_per_sm;
+    int64_t opt_verify_waves;       // grid = waves x the resident capacity (experiments)
     int64_t opt_sample_tiles_per_warp;
     int64_t opt_pdl;                // launch with programmatic stream serialization
 

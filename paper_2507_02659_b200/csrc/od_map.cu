@@ -43,6 +43,8 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
 {
     __shared__ int32_t s_ids[OD_MAX_K];
     __shared__ int32_t s_hit[OD_MAX_K][OD_NGRAM_MAX + 1];   // [offset][length] -> target or -1
+    __shared__ int32_t s_direct[OD_MAX_K];                  // direct map of the id at each offset, or -1
+    __shared__ float s_q[OD_MAX_K];                         // q(d) of each offset
 
     // under programmatic dependent launch: wait for everything earlier in the
     // stream first, only then let the verification kernel start its prefetch
@@ -60,6 +62,12 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
 
     const int s = warp;
     if (s < K) {
+        // what the serial walk below would otherwise fetch one position at a time
+        if (lane == 0) {
+            const int32_t id = s_ids[s];
+            s_direct[s] = (id >= 0 && id < v_q) ? __ldg(vocab_map + id) : -1;
+            s_q[s] = q_sel[(size_t)b * K_max + s];
+        }
         int32_t hit[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
         if (cap > 0) {
             const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
@@ -102,8 +110,8 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
             for (int len = OD_NGRAM_MAX; len >= 2; --len)
                 if (pos + len <= K && s_hit[pos][len] >= 0) { L = len; t = s_hit[pos][len]; break; }
             if (L) {
-                float prod = q_sel[o + pos];
-                for (int j = 1; j < L; ++j) prod *= q_sel[o + pos + j];
+                float prod = s_q[pos];
+                for (int j = 1; j < L; ++j) prod *= s_q[pos + j];
                 tgt_ids[o + m] = t; q_prime[o + m] = prod;
                 span_start[o + m] = pos; span_len[o + m] = L;
                 ++m; pos += L; ++hits;
@@ -112,9 +120,9 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
             const int32_t id = s_ids[pos];
             const bool in_vocab = id >= 0 && id < v_q;
             if (!in_vocab) ++invalid;
-            const int32_t direct = in_vocab ? __ldg(vocab_map + id) : -1;
+            const int32_t direct = s_direct[pos];
             if (direct >= 0) {
-                tgt_ids[o + m] = direct; q_prime[o + m] = q_sel[o + pos];
+                tgt_ids[o + m] = direct; q_prime[o + m] = s_q[pos];
                 span_start[o + m] = pos; span_len[o + m] = 1;
                 ++m; ++pos;
             } else {

@@ -10,16 +10,17 @@
 // blocks, whatever the mix of row counts. The unit of work is 512 contiguous
 // bytes of a row; a row has W units; the rows to read are laid end to end in
 // two flat index spaces and every block takes one contiguous span of each:
-//   space A  row 0 of every sequence. It is always read, so its split needs
-//            nothing from the device: a block asks the copy engine to pull its
-//            span into L2 (cp.async.bulk.prefetch) before it waits for the
-//            translation kernel (programmatic dependent launch) and before it
-//            builds the prefix sums of m, so HBM is busy during both;
+//   space A  row 0 of every sequence. It is always read and its split needs
+//            nothing from the device, so a block works through its span
+//            before it waits for the translation kernel (programmatic
+//            dependent launch): that kernel, and the previous launch's decide
+//            kernel, are hidden behind useful traffic;
 //   space B  rows 1..m_b, split by the prefix sums of m, which every block
 //            rebuilds in shared memory (at most 2048 sequences per launch).
-// A span is cut at row ends into segments; a block reduces a segment to one
-// partial (reference exponent c, sum of exp2(x*scale - c), exact maximum) and
-// stores it. No atomics, no fences, no block waits for another.
+// A span is cut at row ends into segments; every warp of the block reduces its
+// share of a segment to one partial (reference exponent c, sum of
+// exp2(x*scale - c), exact maximum) and stores it. No atomics, no fences, no
+// barriers: no warp waits for another.
 //
 // (2) od_verify_decide_kernel: one block per sequence, one warp per row. Before
 // it waits for the stream kernel it loads what does not depend on it (m, T,
@@ -44,6 +45,10 @@ namespace {
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
 constexpr int U = 4;                            // 16-byte loads in flight per thread
+constexpr int A_PARK = 8;                       // partials of space A a block can hold back
+#ifndef OD_VERIFY_MAXNREG
+#define OD_VERIFY_MAXNREG 56
+#endif
 #ifndef OD_VERIFY_BLOCKS_PER_SM
 #define OD_VERIFY_BLOCKS_PER_SM 4               // resident blocks per SM the register budget allows
 #endif
@@ -54,8 +59,9 @@ struct VerifyArgs {
     int32_t B, K_max, v_p;
     int32_t W;                          // 512-byte units per row
     int32_t n_chunks;                   // blocks of the stream grid
-    int32_t span_min;                   // keeps a row within OD_VERIFY_SEG_MAX segments
+    int32_t span_min;                   // keeps a row within OD_VERIFY_SEG_MAX / WARPS block segments
     int32_t span_a;                     // units of space A per block
+    int32_t a_early;                    // 1: a block's span of space A has at most A_PARK segments
     const int32_t *tgt_ids;
     const float *q_prime;
     const int32_t *span_len;
@@ -91,12 +97,6 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
     return v;
-}
-
-// one thread asks the copy engine to pull [p, p + bytes) into L2 (both multiples of 16)
-__device__ __forceinline__ void l2_prefetch_bulk(const void *p, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
@@ -239,10 +239,10 @@ __device__ __forceinline__ void warp_merge(float &c, float &s, float &mx)
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
 }
 
-// Units [v0, v1) of row (b, r) by the whole block; the partial goes to slot `seg` of the row.
+// Units [v0, v1) of row (b, r) by the whole block; warp w stores its partial to dst[w]
+// (global or shared memory).
 template <int DTYPE>
-__device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r, int seg, int v0, int v1,
-                                              float4 *s_red)
+__device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r, int v0, int v1, float4 *dst)
 {
     constexpr int VEC = DTYPE == OD_BF16 ? 8 : 4;          // elements per 16 bytes
     constexpr size_t ESZ = DTYPE == OD_BF16 ? 2 : 4;
@@ -261,11 +261,27 @@ __device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r,
     const int v1f = v1 < full_units ? v1 : full_units;
     int v = v0 + warp;
     const uint4 *p = (const uint4 *)row + (size_t)v * 32 + lane;
-    for (; v + (U - 1) * WARPS < v1f; v += U * WARPS, p += U * WARPS * 32) {
-        uint4 x[U];
+    // Software pipeline over groups of U units: the loads of the next group are
+    // issued before the current group is folded in, so a warp always has loads in
+    // flight while it keeps the exp pipe busy (warps of a block move in lockstep,
+    // they cannot hide one another's latency).
+    if (v + (U - 1) * WARPS < v1f) {
+        uint4 xa[U], xb[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) x[u] = ld_stream(p + u * WARPS * 32);
-        absorb<DTYPE, U>(L, x, scale);
+        for (int u = 0; u < U; ++u) xa[u] = ld_stream(p + u * WARPS * 32);
+        v += U * WARPS; p += U * WARPS * 32;
+        for (;;) {
+            if (!(v + (U - 1) * WARPS < v1f)) { absorb<DTYPE, U>(L, xa, scale); break; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) xb[u] = ld_stream(p + u * WARPS * 32);
+            v += U * WARPS; p += U * WARPS * 32;
+            absorb<DTYPE, U>(L, xa, scale);
+            if (!(v + (U - 1) * WARPS < v1f)) { absorb<DTYPE, U>(L, xb, scale); break; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) xa[u] = ld_stream(p + u * WARPS * 32);
+            v += U * WARPS; p += U * WARPS * 32;
+            absorb<DTYPE, U>(L, xb, scale);
+        }
     }
     if (v < v1f) {
         const int left = (v1f - v + WARPS - 1) / WARPS;    // 1..U-1, the same for the whole warp
@@ -296,28 +312,28 @@ __device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r,
         const int e = full_vecs * VEC + lane;
         if (e < a.v_p) absorb_one<DTYPE>(L, od_load_logit<DTYPE>(row, e), scale);
     }
+    // every warp publishes its own partial: no block barrier anywhere in the stream
     float c = L.c, s = L.s, mx = L.max_seen();
     warp_merge(c, s, mx);
-    __syncthreads();                                        // s_red may still be read from the last segment
-    if (lane == 0) s_red[warp] = make_float4(c, s, mx, 0.f);
-    __syncthreads();
-    if (warp == 0) {
-        float4 t = lane < WARPS ? s_red[lane] : make_float4(-FLT_MAX, 0.f, -INFINITY, 0.f);
-        c = t.x; s = t.y; mx = t.z;
-        warp_merge(c, s, mx);
-        if (lane == 0)
-            a.partials[((size_t)b * (a.K_max + 1) + r) * OD_VERIFY_SEG_MAX + seg] = make_float4(c, s, mx, 0.f);
-    }
+    if (lane == 0) dst[warp] = make_float4(c, s, mx, 0.f);
 }
 
+// first of the WARPS partial slots of segment `seg` of row (b, r)
+__device__ __forceinline__ float4 *partial_slot(const VerifyArgs &a, int b, int r, int seg)
+{
+    return a.partials + ((size_t)b * (a.K_max + 1) + r) * OD_VERIFY_SEG_MAX + seg * WARPS;
+}
+
+// 56 registers, not 64: four resident blocks then leave an eighth of the SM's register
+// file free, enough for a block of the (small) kernel before or after this one in
+// the stream to be resident at the same time under programmatic dependent launch.
 template <int DTYPE>
-__global__ void __launch_bounds__(THREADS, OD_VERIFY_BLOCKS_PER_SM)
+__global__ void __maxnreg__(OD_VERIFY_MAXNREG)
 od_verify_stream_kernel(const VerifyArgs a)
 {
-    constexpr size_t ESZ = DTYPE == OD_BF16 ? 2 : 4;
     __shared__ int32_t s_cum[OD_VERIFY_MAX_B + 1];          // exclusive prefix of the clamped m_b
     __shared__ int32_t s_wsum[WARPS];
-    __shared__ float4 s_red[WARPS];
+    __shared__ float4 s_park[A_PARK][WARPS];
 
     // Flat unit indices fit 32 bits (the launcher checks): the walk below is
     // executed by every thread, so it uses 32-bit arithmetic and as few
@@ -326,28 +342,31 @@ od_verify_stream_kernel(const VerifyArgs a)
     const uint32_t g = blockIdx.x;
     const uint32_t W = (uint32_t)a.W;
 
-    // ---- space A (row 0 of every sequence): ask for this block's bytes before anything else
+    // ---- space A (row 0 of every sequence). Nothing here depends on the translation
+    // kernel (logits and temperatures are inputs of the step), so under programmatic
+    // dependent launch this phase runs while that kernel is still at work. Its partials
+    // wait in shared memory: the scratch in global memory may still be read by the
+    // previous launch's decide kernel until griddepcontrol.wait returns.
     const uint32_t a_tot = (uint32_t)a.B * W;
     uint32_t a_lo = g * (uint32_t)a.span_a;
     if (a_lo > a_tot) a_lo = a_tot;
     uint32_t a_hi = a_lo + (uint32_t)a.span_a;
     if (a_hi > a_tot) a_hi = a_tot;
     const uint32_t a_b0 = a_lo / W, a_v0 = a_lo - a_b0 * W;   // first sequence and unit of the span
-    if (threadIdx.x == 0 && a_lo < a_hi) {
-        const uint32_t row_bytes16 = (uint32_t)((size_t)a.v_p * ESZ / 16 * 16);
+    const uint32_t a_seg0 = g - (a_lo - a_v0) / (uint32_t)a.span_a;   // a row that starts here has segment 0 here
+    const bool early = a.a_early != 0;                      // the span has at most A_PARK segments
+    if (early && a_lo < a_hi) {
         uint32_t f = a_lo, b = a_b0, v0 = a_v0;
+        int k = 0;
         while (f < a_hi) {
             uint32_t n = a_hi - f;
             if (n > W - v0) n = W - v0;
-            const char *row = (const char *)a.logits + (size_t)b * a.seq_stride * ESZ;
-            uint32_t lo = v0 * 512u, hi = (v0 + n) * 512u;
-            if (hi > row_bytes16) hi = row_bytes16;
-            if (hi > lo) l2_prefetch_bulk(row + lo, hi - lo);
+            block_segment<DTYPE>(a, (int)b, 0, (int)v0, (int)(v0 + n), s_park[k++]);
             f += n; ++b; v0 = 0;
         }
     }
 
-    // everything below may read what the translation kernel wrote
+    // everything below may read what the translation kernel wrote, and may write scratch
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
 
@@ -376,15 +395,26 @@ od_verify_stream_kernel(const VerifyArgs a)
         __syncthreads();
     }
 
-    // ---- space A: a row that starts inside this span has its segment 0 here
     if (a_lo < a_hi) {
-        uint32_t f = a_lo, b = a_b0, v0 = a_v0;
-        uint32_t seg = g - (a_lo - a_v0) / (uint32_t)a.span_a;
-        while (f < a_hi) {
-            uint32_t n = a_hi - f;
-            if (n > W - v0) n = W - v0;
-            block_segment<DTYPE>(a, (int)b, 0, (int)seg, (int)v0, (int)(v0 + n), s_red);
-            f += n; ++b; v0 = 0; seg = 0;
+        if (early) {
+            // hand the parked partials over (the barriers above made them visible)
+            uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
+            int k = 0;
+            while (f < a_hi) {
+                uint32_t n = a_hi - f;
+                if (n > W - v0) n = W - v0;
+                if (warp == (k & (WARPS - 1)) && lane < WARPS)
+                    partial_slot(a, (int)b, 0, (int)seg)[lane] = s_park[k][lane];
+                ++k; f += n; ++b; v0 = 0; seg = 0;
+            }
+        } else {
+            uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
+            while (f < a_hi) {
+                uint32_t n = a_hi - f;
+                if (n > W - v0) n = W - v0;
+                block_segment<DTYPE>(a, (int)b, 0, (int)v0, (int)(v0 + n), partial_slot(a, (int)b, 0, (int)seg));
+                f += n; ++b; v0 = 0; seg = 0;
+            }
         }
     }
 
@@ -413,7 +443,8 @@ od_verify_stream_kernel(const VerifyArgs a)
             while ((uint32_t)s_cum[b + 1] <= rho) ++b;
             uint32_t n = f_hi - f;
             if (n > W - v0) n = W - v0;
-            block_segment<DTYPE>(a, b, 1 + (int)(rho - (uint32_t)s_cum[b]), (int)seg, (int)v0, (int)(v0 + n), s_red);
+            const int r = 1 + (int)(rho - (uint32_t)s_cum[b]);
+            block_segment<DTYPE>(a, b, r, (int)v0, (int)(v0 + n), partial_slot(a, b, r, (int)seg));
             f += n; ++rho; v0 = 0; seg = 0;
         }
     }
@@ -482,7 +513,7 @@ od_verify_decide_kernel(const VerifyArgs a)
         const int row_slot = b * (a.K_max + 1) + r;
         const float4 *pp = a.partials + (size_t)row_slot * OD_VERIFY_SEG_MAX;
         float c = -FLT_MAX, s = 0.f, mx = -INFINITY;
-        for (int k = lane; k < nseg; k += 32) {
+        for (int k = lane; k < nseg * WARPS; k += 32) {
             const float4 p = __ldcg(pp + k);
             pair_merge(c, s, p.x, p.y);
             mx = fmaxf(mx, p.z);
@@ -552,7 +583,9 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
     const int64_t row_bytes = (int64_t)c->v_p * esz;
     const int32_t W = (int32_t)((row_bytes + 511) / 512);
-    const int32_t span_min = (W + OD_VERIFY_SEG_MAX - 2) / (OD_VERIFY_SEG_MAX - 1);
+    // a row is cut into at most OD_VERIFY_SEG_MAX / WARPS block segments (one partial per warp each)
+    constexpr int MAX_BLOCK_SEGS = OD_VERIFY_SEG_MAX / WARPS;
+    const int32_t span_min = (W + MAX_BLOCK_SEGS - 2) / (MAX_BLOCK_SEGS - 1);
     int64_t blocks_per_sm = c->opt_verify_blocks_per_sm > 0 ? c->opt_verify_blocks_per_sm : OD_VERIFY_BLOCKS_PER_SM;
     if (blocks_per_sm > OD_VERIFY_BLOCKS_PER_SM) blocks_per_sm = OD_VERIFY_BLOCKS_PER_SM;
 
@@ -564,7 +597,7 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
         const int32_t nb = B - b0 < slice ? B - b0 : slice;
         // no more blocks than the most this slice can need
         const int64_t max_units = (int64_t)nb * (K_max + 1) * W;
-        int64_t grid = (int64_t)c->sm_count * blocks_per_sm;
+        int64_t grid = (int64_t)c->sm_count * blocks_per_sm * (c->opt_verify_waves > 0 ? c->opt_verify_waves : 1);
         const int64_t need = max_units / span_min + 1;
         if (grid > need) grid = need;
         if (grid < 1) grid = 1;
@@ -576,6 +609,7 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
         int64_t span_a = ((int64_t)nb * W + grid - 1) / grid;
         if (span_a < span_min) span_a = span_min;
         a.span_a = (int32_t)span_a;
+        a.a_early = span_a / W + 2 <= A_PARK;
         a.tgt_ids = tgt_ids + (size_t)b0 * K_max; a.q_prime = q_prime + (size_t)b0 * K_max;
         a.span_len = span_len + (size_t)b0 * K_max; a.m = m + b0;
         a.temperature = temperature + b0; a.seed = seed + b0; a.step = step;
