@@ -1,6 +1,7 @@
 // C ABI of the library (see include/omnidraft.h): context life cycle, the
 // host-side builds of the vocabulary map and of the n-gram cache table,
 // argument validation, and the whole-step entry point for host buffers.
+#include <algorithm>
 #include <new>
 #include <string.h>
 #include <vector>
@@ -43,7 +44,7 @@ int32_t dev_alloc(T **p, size_t n)
 
 void free_all(od_ctx *c)
 {
-    void *ptrs[] = {c->d_vocab_map, c->d_inv_map, c->d_keys, c->d_vals, c->d_partials,
+    void *ptrs[] = {c->d_vocab_map, c->d_inv_map, c->d_mapped_t, c->d_mapped_d, c->d_keys, c->d_vals, c->d_partials,
                     c->d_tile_sums,
                     c->d_samp_ticket, c->s_logits, c->s_q_rows, c->s_q_sel, c->s_temperature,
                     c->s_draft_ids, c->s_draft_len, c->s_seed, c->s_tgt_ids, c->s_span_start,
@@ -112,6 +113,7 @@ int32_t od_create(od_ctx **ctx, int32_t device, int32_t draft_vocab, int32_t tar
     int32_t st = OD_OK;
     if (st == OD_OK) st = dev_alloc(&c->d_vocab_map, (size_t)draft_vocab);
     if (st == OD_OK) st = dev_alloc(&c->d_inv_map, (size_t)target_vocab + 8);
+
     if (st == OD_OK) st = dev_alloc(&c->d_partials, rows * OD_VERIFY_SEG_MAX);
     if (st == OD_OK) st = dev_alloc(&c->d_tile_sums, (size_t)max_batch * c->tiles_per_row);
     if (st == OD_OK) st = dev_alloc(&c->d_samp_ticket, (size_t)max_batch);
@@ -153,6 +155,31 @@ int32_t od_set_vocab_map(od_ctx *c, const int32_t *host_map)
     for (int32_t d = 0; d < c->v_q; ++d) fwd[d] = host_map[d] < 0 ? -1 : host_map[d];
     OD_CUDA(cudaMemcpy(c->d_vocab_map, fwd.data(), fwd.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
     OD_CUDA(cudaMemcpy(c->d_inv_map, inv.data(), inv.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    // the same inverse map as one fixed-width list per tile of target ids (for the residual sampler)
+    const size_t ntiles = (size_t)c->tiles_per_row;
+    std::vector<int32_t> count(ntiles, 0);
+    for (int32_t t = 0; t < c->v_p; ++t)
+        if (inv[t] >= 0) ++count[t / OD_SAMPLE_TILE];
+    int32_t longest = 1;
+    for (size_t i = 0; i < ntiles; ++i) longest = count[i] > longest ? count[i] : longest;
+    const int32_t width = (longest + 31) / 32 * 32;
+    std::vector<int32_t> mt(ntiles * width, -1), md(ntiles * width, 0);
+    std::fill(count.begin(), count.end(), 0);
+    for (int32_t t = 0; t < c->v_p; ++t) {
+        if (inv[t] < 0) continue;
+        const size_t i = (size_t)t / OD_SAMPLE_TILE;
+        mt[i * width + count[i]] = t;
+        md[i * width + count[i]] = inv[t];
+        ++count[i];
+    }
+    if (c->d_mapped_t) { cudaFree(c->d_mapped_t); c->d_mapped_t = nullptr; }
+    if (c->d_mapped_d) { cudaFree(c->d_mapped_d); c->d_mapped_d = nullptr; }
+    int32_t st = dev_alloc(&c->d_mapped_t, mt.size());
+    if (st == OD_OK) st = dev_alloc(&c->d_mapped_d, md.size());
+    if (st != OD_OK) return st;
+    OD_CUDA(cudaMemcpy(c->d_mapped_t, mt.data(), mt.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    OD_CUDA(cudaMemcpy(c->d_mapped_d, md.data(), md.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    c->list_width = width;
     c->have_map = true;
     return OD_OK;
 }

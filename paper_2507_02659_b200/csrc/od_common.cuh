@@ -23,6 +23,12 @@ struct od_ctx {
     // vocabulary map (device)
     int32_t *d_vocab_map;           // [v_q]
     int32_t *d_inv_map;             // [v_p], -1 outside the image
+    // the mapped ids sorted by target id, as one fixed-width list per tile of
+    // OD_SAMPLE_TILE target ids: entry k of tile i is at i * list_width + k,
+    // unused entries hold target id -1 (and draft id 0)
+    int32_t *d_mapped_t;            // [tiles_per_row * list_width] target id
+    int32_t *d_mapped_d;            // [tiles_per_row * list_width] its draft id
+    int32_t list_width;             // multiple of 32, >= the longest list
     bool have_map;
 
     // n-gram cache: open addressing over groups of 32 slots
@@ -34,7 +40,7 @@ struct od_ctx {
     float4 *d_partials;             // [rows][OD_VERIFY_SEG_MAX] (c, sum, max, -), rows of one launch
 
     // od_sample_residual scratch
-    double *d_tile_sums;            // [max_batch * tiles_per_row]
+    double *d_tile_sums;            // [max_batch * tiles_per_row] value of each tile
     unsigned int *d_samp_ticket;    // [max_batch]
     int32_t tiles_per_row;
 
@@ -136,6 +142,37 @@ __device__ __forceinline__ float od_ex2(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Packed fp32 pairs (one instruction for two lanes of arithmetic on sm_100).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// acc += (exp2(lo*scale - c), exp2(hi*scale - c))
+__device__ __forceinline__ uint64_t f2_exp_acc(uint64_t acc, float lo, float hi, uint64_t scale2, uint64_t nc2)
+{
+    float e0, e1;
+    f2_unpack(f2_fma(f2_pack(lo, hi), scale2, nc2), e0, e1);
+    return f2_add(acc, f2_pack(od_ex2(e0), od_ex2(e1)));
 }
 
 // (max, sum) of exp2((x - max) * scale): merge two partial pairs

@@ -5,17 +5,28 @@
 // free-token lines).
 //
 // Inverse-CDF sampling in target-id order over tiles of 256 ids (8 consecutive
-// ids per lane of one warp, so a tile needs shuffles only, no block barrier):
-//   pass 1  every warp computes r(t) for its run of tiles of row j = n_b and
-//           stores one fp64 sum per tile;
+// ids per lane of one warp, so a tile needs shuffles only, no block barrier).
+// Values are carried unnormalised: e(t) = exp2((x_t - M)*scale) = p(t)*S and
+// r'(t) = max(0, e(t) - q'(t)*S) = e(t) - min(e(t), q'(t)*S), so that
+//   sum over a tile of r' = (sum of e over the tile) - (sum over the mapped ids t
+//   of the tile of min(e(t), q'(t)*S)).
+// Only a sixth of the target ids have a draft pre-image, and the context holds them
+// sorted by target id as one fixed-width list per tile, so:
+//   pass 1  every warp takes a run of tiles of row j = n_b; per tile it sums e over
+//           the 256 ids (coalesced 128-bit loads) minus the corrections over the tile's
+//           list (a coalesced read of the list, one gathered drafter probability and
+//           one logit, already in cache, per entry) and stores the tile's value;
 //   ticket  blocks never wait for each other: the block that draws the
 //           sequence's last ticket continues alone;
-//   pass 2  that block scans the tile sums in parallel (R = total, target =
-//           u * R), finds the tile in which the running sum crosses the target,
-//           and one warp recomputes that tile (L2-resident) and scans inside it.
-// r(t) is evaluated in fp32 exactly the same way in both passes; all sums and
-// scans are fp64 in a fixed order, so the result is reproducible and the only
-// difference to exact arithmetic is the fp32 rounding of the individual r(t).
+//   pass 2  that block scans the tile values in parallel (total,
+//           target = u * total), finds the tile in which the running sum crosses
+//           the target, and one warp evaluates r'(t) of that single tile id by id
+//           (through the inverse map, with the two ids Eq. (2) singles out) and
+//           scans inside it. Without residual mass it draws from p_j (it then
+//           redoes the tile sums with e alone).
+// Sums and scans across lanes and tiles are fp64 in a fixed order: the result is
+// reproducible, and the only difference to exact arithmetic is the fp32 rounding
+// of the individual terms.
 #include <float.h>
 
 #include "od_common.cuh"
@@ -43,7 +54,9 @@ struct SampleArgs {
     int32_t *out_token;
     float *resid_mass;
     uint32_t *flags;
-    double *tile_sums;
+    const int32_t *mapped_t, *mapped_d;   // mapped ids: one list of list_width entries per tile
+    int32_t list_width;
+    double *tile_val;                   // [B][ntiles] sum over the tile of r'
     unsigned int *ticket;
 };
 
@@ -51,20 +64,22 @@ struct SampleArgs {
 struct SeqState {
     const char *row;
     const float *q_row;
-    float M, S, scale;
+    float c, S, scale;      // e(t) = exp2(fma(x_t, scale, -c)); S is the row sum relative to c
     bool residual;
-    int32_t ngram_token, prefix_token;
+    int32_t ngram_token, prefix_token, first_draft;
     float ngram_prob, prefix_val;
 };
 
-// Values are carried UNNORMALISED: with e(t) = exp2((x_t - M)*scale) = p(t)*S,
+// Values are carried UNNORMALISED: with c = fl(M*scale), e(t) = exp2(x_t*scale - c) and
+// S = (row sum relative to M) * exp2(M*scale - c), so that p(t) = e(t)/S exactly as
+// before but one fused multiply-add per id replaces a subtraction and a product,
 //   residual   r'(t) = max(0, e(t) - q'(t)*S) = S * max(0, p(t) - q'(t))
 //   free token r'(t) = e(t)
 // so one multiplication by 1/S at the very end replaces one per element, and the
 // inverse-CDF pick (target = u * sum r') is unchanged by the common factor.
 __device__ __forceinline__ float resid_of(const SeqState &q, float x, float qq)
 {
-    return fmaxf(0.f, fmaf(-qq, q.S, od_ex2((x - q.M) * q.scale)));
+    return fmaxf(0.f, fmaf(-qq, q.S, od_ex2(fmaf(x, q.scale, -q.c))));
 }
 
 // r'(t) of the EPT consecutive ids this lane owns in `tile`; ids >= v_p give 0
@@ -96,7 +111,7 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
             for (int e = 0; e < EPT; ++e) r[e] = resid_of(q, x[e], qq[e]);
         } else {
 #pragma unroll
-            for (int e = 0; e < EPT; ++e) r[e] = od_ex2((x[e] - q.M) * q.scale);
+            for (int e = 0; e < EPT; ++e) r[e] = od_ex2(fmaf(x[e], q.scale, -q.c));
         }
     } else {
 #pragma unroll
@@ -109,7 +124,7 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
                     const int32_t dv = __ldg(a.inv_map + t);
                     r[e] = resid_of(q, xv, dv >= 0 ? __ldg(q.q_row + dv) : 0.f);
                 } else {
-                    r[e] = od_ex2((xv - q.M) * q.scale);
+                    r[e] = od_ex2(fmaf(xv, q.scale, -q.c));
                 }
             }
         }
@@ -141,46 +156,172 @@ __device__ __forceinline__ double lane_sum(const float *r)
     return (double)s;
 }
 
-__device__ __forceinline__ double warp_sum(double v)
+// e(t) of the EPT consecutive ids this lane owns in `tile`; ids >= v_p give 0
+template <int DTYPE>
+__device__ __forceinline__ void tile_e_values(const SeqState &q, const SampleArgs &a, int tile, int lane, float *r)
+{
+    const int t0 = tile * OD_SAMPLE_TILE + lane * EPT;
+    if (t0 + EPT <= a.v_p) {
+        float x[EPT];
+        if (DTYPE == OD_BF16) {
+            const uint4 v = __ldg((const uint4 *)(q.row + (size_t)t0 * 2));
+            x[0] = od_bf16_lo(v.x); x[1] = od_bf16_hi(v.x); x[2] = od_bf16_lo(v.y); x[3] = od_bf16_hi(v.y);
+            x[4] = od_bf16_lo(v.z); x[5] = od_bf16_hi(v.z); x[6] = od_bf16_lo(v.w); x[7] = od_bf16_hi(v.w);
+        } else {
+            const float4 v0 = __ldg((const float4 *)(q.row + (size_t)t0 * 4));
+            const float4 v1 = __ldg((const float4 *)(q.row + (size_t)t0 * 4) + 1);
+            x[0] = v0.x; x[1] = v0.y; x[2] = v0.z; x[3] = v0.w;
+            x[4] = v1.x; x[5] = v1.y; x[6] = v1.z; x[7] = v1.w;
+        }
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) r[e] = od_ex2(fmaf(x[e], q.scale, -q.c));
+    } else {
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) {
+            const int t = t0 + e;
+            r[e] = t < a.v_p ? od_ex2(fmaf(od_load_logit<DTYPE>(q.row, t), q.scale, -q.c)) : 0.f;
+        }
+    }
+}
+
+// one entry of a tile's list: min(e(t), q'(t)*S). The id that Eq. (2) gives the
+// n-gram's probability is left to the caller; the first sub-token of the n-gram
+// carries the reduced probability.
+template <int DTYPE>
+__device__ __forceinline__ float corr_term(const SeqState &q, int32_t t, int32_t d, float x, float qd)
+{
+    if (t < 0 || t == q.ngram_token) return 0.f;
+    if (d == q.first_draft) qd = q.prefix_val;
+    return fminf(od_ex2(fmaf(x, q.scale, -q.c)), qd * q.S);
+}
+
+__device__ __forceinline__ float warp_sum_f32(float v)
 {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
     return v;
 }
 
-// tile sums of tiles [t_lo, t_hi) by one warp: index order inside a lane, xor
-// tree across the lanes
-template <int DTYPE>
-__device__ __forceinline__ void warp_tiles(const SeqState &q, const SampleArgs &a, bool residual,
-                                           int t_lo, int t_hi, int lane, double *sums)
+// pass 1 for a batch of n <= TB consecutive tiles by one warp: the value of a tile is
+// (sum of e over its ids) - (sum of the corrections over its list). A lane adds its
+// eight e's and subtracts the corrections of the list entries it is given (lane l
+// takes entries l, l + 32, ... of the tile's list), so ONE warp sum per tile yields
+// the tile's value. This pass is bound by instruction issue and memory latency, not
+// by bandwidth: the loads of the whole batch are issued level by level (logits and
+// list bounds, then list entries, then the gathered probabilities and logits).
+template <int DTYPE, int TB>
+__device__ __forceinline__ void warp_batch(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
+                                           int n, int lane, double *tile_val)
 {
-    int tile = t_lo;
-    for (; tile + 2 <= t_hi; tile += 2) {                  // two tiles in flight
-        float r0[EPT], r1[EPT];
-        tile_values<DTYPE>(q, a, residual, tile, lane, r0);
-        tile_values<DTYPE>(q, a, residual, tile + 1, lane, r1);
-        const double s0 = warp_sum(lane_sum(r0)), s1 = warp_sum(lane_sum(r1));
-        if (lane == 0) { sums[tile] = s0; sums[tile + 1] = s1; }
+    uint4 raw[TB][DTYPE == OD_BF16 ? 1 : 2];
+    const int whole_n = (a.v_p / OD_SAMPLE_TILE - t_lo) < n ? (a.v_p / OD_SAMPLE_TILE - t_lo) : n;   // tiles with all 256 ids
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+        if (i < whole_n) {
+            const uint4 *src = (const uint4 *)(q.row + ((size_t)(t_lo + i) * OD_SAMPLE_TILE + lane * EPT) *
+                                                           (DTYPE == OD_BF16 ? 2 : 4));
+            raw[i][0] = __ldg(src);
+            if (DTYPE != OD_BF16) raw[i][1] = __ldg(src + 1);
+        }
     }
-    if (tile < t_hi) {
-        float r0[EPT];
-        tile_values<DTYPE>(q, a, residual, tile, lane, r0);
-        const double s0 = warp_sum(lane_sum(r0));
-        if (lane == 0) sums[tile] = s0;
+    // the first two rounds of every tile's list (its address needs no lookup: fixed width;
+    // unused entries hold -1); wider lists finish below
+    int32_t et[TB][2], ed[TB][2];
+    const int rounds = a.list_width >> 5;
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const bool ok = residual && i < n && k < rounds;
+            const size_t idx = (size_t)(t_lo + i) * a.list_width + k * 32 + lane;
+            et[i][k] = ok ? __ldg(a.mapped_t + idx) : -1;
+            ed[i][k] = ok ? __ldg(a.mapped_d + idx) : 0;
+        }
     }
-    __threadfence();                                       // the sums are read by another block
+    float ex[TB][2], eq[TB][2];
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int32_t t = et[i][k] >= 0 ? et[i][k] : 0;   // always a valid address; the term is dropped below
+            ex[i][k] = od_load_logit<DTYPE>(q.row, t);
+            eq[i][k] = __ldg(q.q_row + ed[i][k]);
+        }
+    }
+
+    const uint64_t scale2 = f2_pack(q.scale, q.scale), nc2 = f2_pack(-q.c, -q.c);
+    float mine = 0.f;
+#pragma unroll
+    for (int i = 0; i < TB; ++i) {
+        if (i < n) {                                        // n and whole_n are the same for the whole warp
+            float sum;
+            if (i < whole_n) {
+                uint64_t acc = 0ull;
+                if (DTYPE == OD_BF16) {
+                    const uint4 v = raw[i][0];
+                    acc = f2_exp_acc(acc, od_bf16_lo(v.x), od_bf16_hi(v.x), scale2, nc2);
+                    acc = f2_exp_acc(acc, od_bf16_lo(v.y), od_bf16_hi(v.y), scale2, nc2);
+                    acc = f2_exp_acc(acc, od_bf16_lo(v.z), od_bf16_hi(v.z), scale2, nc2);
+                    acc = f2_exp_acc(acc, od_bf16_lo(v.w), od_bf16_hi(v.w), scale2, nc2);
+                } else {
+                    const uint4 v0 = raw[i][0], v1 = raw[i][DTYPE == OD_BF16 ? 0 : 1];
+                    acc = f2_exp_acc(acc, __uint_as_float(v0.x), __uint_as_float(v0.y), scale2, nc2);
+                    acc = f2_exp_acc(acc, __uint_as_float(v0.z), __uint_as_float(v0.w), scale2, nc2);
+                    acc = f2_exp_acc(acc, __uint_as_float(v1.x), __uint_as_float(v1.y), scale2, nc2);
+                    acc = f2_exp_acc(acc, __uint_as_float(v1.z), __uint_as_float(v1.w), scale2, nc2);
+                }
+                float s0, s1;
+                f2_unpack(acc, s0, s1);
+                sum = s0 + s1;
+            } else {
+                float r[EPT];
+                tile_e_values<DTYPE>(q, a, t_lo + i, lane, r);   // the ragged last tile, id by id
+                sum = r[0];
+#pragma unroll
+                for (int e = 1; e < EPT; ++e) sum += r[e];
+            }
+            if (residual) {
+#pragma unroll
+                for (int k = 0; k < 2; ++k) sum -= corr_term<DTYPE>(q, et[i][k], ed[i][k], ex[i][k], eq[i][k]);
+                for (int k = 2; k < rounds; ++k) {              // a wide list
+                    const size_t idx = (size_t)(t_lo + i) * a.list_width + k * 32 + lane;
+                    const int32_t t = __ldg(a.mapped_t + idx), d = __ldg(a.mapped_d + idx);
+                    sum -= corr_term<DTYPE>(q, t, d, od_load_logit<DTYPE>(q.row, t >= 0 ? t : 0), __ldg(q.q_row + d));
+                }
+                // the n-gram's own token carries the n-gram's probability
+                if (lane == 0 && q.ngram_token >= 0 && q.ngram_token < a.v_p &&
+                    q.ngram_token / OD_SAMPLE_TILE == t_lo + i)
+                    sum -= fminf(od_ex2(fmaf(od_load_logit<DTYPE>(q.row, q.ngram_token), q.scale, -q.c)),
+                                 q.ngram_prob * q.S);
+            }
+            sum = warp_sum_f32(sum);
+            if (lane == i) mine = sum;
+        }
+    }
+    if (lane < n) tile_val[t_lo + lane] = (double)mine;
+}
+
+template <int DTYPE>
+__device__ __forceinline__ void warp_tiles(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
+                                           int t_hi, int lane, double *tile_val)
+{
+    constexpr int TB = 4;
+    for (int t = t_lo; t < t_hi; t += TB)
+        warp_batch<DTYPE, TB>(q, a, residual, t, t_hi - t < TB ? t_hi - t : TB, lane, tile_val);
 }
 
 template <int DTYPE>
 __global__ void __launch_bounds__(OD_SAMPLE_THREADS, 4)
 od_sample_kernel(const SampleArgs a)
 {
+    extern __shared__ __align__(16) unsigned char s_dyn[];   // ntiles x 8 bytes
+    double *s_val = (double *)s_dyn;                         // pass 2: tile values
     __shared__ double s_warp[WARPS];
     __shared__ unsigned int s_last;
-    __shared__ int s_tile, s_lastmass;
+    __shared__ int s_tile, s_lastmass, s_token;
     __shared__ double s_before, s_total;
 
-    // n_accepted and the row statistics come from the verification kernel
+    // n_accepted and the row statistics come from the verification kernels
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
 
@@ -202,43 +343,58 @@ od_sample_kernel(const SampleArgs a)
     const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
     SeqState q;
     q.row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)j * a.row_stride) * esz;
-    q.M = a.row_max[b * (K + 1) + j];
-    q.S = a.row_sum[b * (K + 1) + j];
     q.scale = 1.4426950408889634f / T;
+    {
+        // reference exponent c = fl(M*scale); the rounding of c goes into S exactly:
+        // sum_t exp2(x_t*scale - c) = (sum_t exp2((x_t - M)*scale)) * exp2(M*scale - c)
+        const float M = a.row_max[b * (K + 1) + j];
+        q.c = fmaxf(M * q.scale, -FLT_MAX);
+        q.S = a.row_sum[b * (K + 1) + j] * od_ex2(fmaf(M, q.scale, -q.c));
+    }
     q.residual = (j < mb) || stop;
-    q.ngram_token = -1; q.prefix_token = -1; q.ngram_prob = 0.f; q.prefix_val = 0.f;
+    q.ngram_token = -1; q.prefix_token = -1; q.first_draft = -1; q.ngram_prob = 0.f; q.prefix_val = 0.f;
     q.q_row = a.q_rows;
     if (q.residual) {
         const size_t o = (size_t)b * K + j;
         int s0 = a.span_start[o];
         s0 = s0 < 0 ? 0 : (s0 >= K ? K - 1 : s0);
         q.q_row = a.q_rows + ((size_t)b * K + s0) * a.v_q;
+        // the gathers of pass 1 come two round trips from now: have the copy engine pull
+        // this block's share of the drafter's row into L2 meanwhile
+        if (threadIdx.x == 0) {
+            const size_t row_bytes = (size_t)a.v_q * 4 / 16 * 16;
+            size_t lo = (row_bytes / gridDim.x * blockIdx.x) / 16 * 16;
+            size_t hi = blockIdx.x + 1 == gridDim.x ? row_bytes : (row_bytes / gridDim.x * (blockIdx.x + 1)) / 16 * 16;
+            const char *base = (const char *)q.q_row;
+            if (((uintptr_t)base & 15u) == 0 && hi > lo)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + lo), "r"((uint32_t)(hi - lo)) : "memory");
+        }
         const int len = j < mb ? a.span_len[o] : 1;
         if (len >= 2) {
             q.ngram_token = a.tgt_ids[o];
             q.ngram_prob = a.q_prime[o];
             const int32_t d1 = a.draft_ids[(size_t)b * K + s0];
             if (d1 >= 0 && d1 < a.v_q) {
+                q.first_draft = d1;
                 q.prefix_token = __ldg(a.vocab_map + d1);
                 q.prefix_val = __ldg(q.q_row + d1) - q.ngram_prob;
             }
         }
     }
 
-    // ---- pass 1: one fp64 sum per tile ----
     const int ntiles = a.ntiles;
-    double *sums = a.tile_sums + (size_t)b * ntiles;
+    double *tile_val = a.tile_val + (size_t)b * ntiles;
+
+    // ---- pass 1: the value of every tile ----
     {
         const int t_lo = (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
         int t_hi = t_lo + a.tiles_per_warp;
         if (t_hi > ntiles) t_hi = ntiles;
-        if (t_lo < t_hi) warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, sums);
+        if (t_lo < t_hi) warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
     }
+    __threadfence();                               // the tile values are read by another block
     __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
-    }
+    if (threadIdx.x == 0) s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
     __syncthreads();
     if (!s_last) return;
     __threadfence();
@@ -250,12 +406,14 @@ od_sample_kernel(const SampleArgs a)
     const int per = (ntiles + OD_SAMPLE_THREADS - 1) / OD_SAMPLE_THREADS;
     const int my_lo = threadIdx.x * per;
     const int my_hi = my_lo + per < ntiles ? my_lo + per : ntiles;
-    const volatile double *vs = sums;
-    double target = 0.0;
+    // tile values (rounding can leave a tile without residual mass slightly negative)
+    for (int t = threadIdx.x; t < ntiles; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, __ldcg(tile_val + t));
+    if (threadIdx.x == 0) a.ticket[b] = 0;
+    __syncthreads();
     for (int attempt = 0; attempt < 2; ++attempt) {
-        // exclusive scan of the tile sums: thread i owns `per` consecutive tiles
+        // exclusive scan of the tile values: thread i owns `per` consecutive tiles
         double loc = 0.0;
-        for (int t = my_lo; t < my_hi; ++t) loc += vs[t];
+        for (int t = my_lo; t < my_hi; ++t) loc += s_val[t];
         double inc = loc;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -263,19 +421,20 @@ od_sample_kernel(const SampleArgs a)
             if (lane >= off) inc += v;
         }
         if (lane == 31) s_warp[warp] = inc;
-        if (threadIdx.x == 0) { s_tile = 0x7FFFFFFF; s_lastmass = -1; }
+        if (threadIdx.x == 0) { s_tile = 0x7FFFFFFF; s_lastmass = -1; s_token = -2; }
         __syncthreads();
         double base = 0.0;
         for (int w = 0; w < warp; ++w) base += s_warp[w];
         if (threadIdx.x == OD_SAMPLE_THREADS - 1) s_total = base + inc;
         __syncthreads();
-        const double R = s_total;
-        if (R > 0.0) {
-            target = (double)u * R;
+        const double Rn = s_total;                  // unnormalised total
+        double target = 0.0;
+        if (Rn > 0.0) {
+            target = (double)u * Rn;
             double c = base + inc - loc;
             int last = -1;
             for (int t = my_lo; t < my_hi; ++t) {
-                const double v = vs[t];
+                const double v = s_val[t];
                 if (v > 0.0) last = t;
                 if (c + v > target) { atomicMin(&s_tile, t); break; }   // first crossing of this run
                 c += v;
@@ -283,90 +442,77 @@ od_sample_kernel(const SampleArgs a)
             if (last >= 0) atomicMax(&s_lastmass, last);
         }
         __syncthreads();
-        if (R > 0.0) {
-            // cumulative sums never decrease, so the smallest reported tile is the crossing;
-            // if rounding hid it, take the last tile that has mass
-            const int t_pick = s_tile != 0x7FFFFFFF ? s_tile : s_lastmass;
-            __syncthreads();
-            if (t_pick >= my_lo && t_pick < my_hi) {        // its owner publishes the sum before it
-                double c = base + inc - loc;
-                for (int t = my_lo; t < t_pick; ++t) c += vs[t];
-                s_before = c;
-                s_tile = t_pick;
+        // cumulative sums never decrease, so the smallest reported tile is the crossing;
+        // if rounding hid it, take the last tile that has mass
+        const int t_pick = Rn > 0.0 ? (s_tile != 0x7FFFFFFF ? s_tile : s_lastmass) : -1;
+        if (t_pick >= my_lo && t_pick < my_hi) {    // its owner publishes the sum before it
+            double c = base + inc - loc;
+            for (int t = my_lo; t < t_pick; ++t) c += s_val[t];
+            s_before = c;
+        }
+        __syncthreads();
+        if (t_pick >= 0 && warp == 0) {
+            // ---- warp 0 evaluates the chosen tile id by id and scans inside it ----
+            float r[EPT];
+            if (residual) tile_values<DTYPE>(q, a, true, t_pick, lane, r);
+            else tile_e_values<DTYPE>(q, a, t_pick, lane, r);
+            const double mine = lane_sum(r);
+            double incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const double v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += v;
             }
-            __syncthreads();
-            break;
+            const double lbase = s_before + (incl - mine);   // sum before this lane's first id
+            const int t0 = t_pick * OD_SAMPLE_TILE + lane * EPT;
+            int my_pick = 0x7FFFFFFF, my_last = -1;
+            double lo = 0.0, hi = 0.0, c = lbase;
+            float run = 0.f;                        // same fp32 order as lane_sum
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) {
+                run = e == 0 ? r[0] : run + r[e];
+                const double nc = lbase + (double)run;
+                if (r[e] > 0.f) my_last = t0 + e;
+                if (my_pick == 0x7FFFFFFF && nc > target) { my_pick = t0 + e; lo = c; hi = nc; }
+                c = nc;
+            }
+            int pick = my_pick, last = my_last;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                pick = min(pick, __shfl_xor_sync(0xFFFFFFFFu, pick, off));
+                last = max(last, __shfl_xor_sync(0xFFFFFFFFu, last, off));
+            }
+            const float R = (float)(Rn / (double)q.S);     // residual mass (1 for the free token)
+            if (pick != 0x7FFFFFFF) {
+                if (my_pick == pick) {              // exactly one lane owns the picked id
+                    uint32_t f = flags;
+                    if (fmin(target - lo, hi - target) <= OD_TAU_SAMPLE * Rn) f |= OD_SF_BOUNDARY;
+                    a.out_token[b] = pick; a.resid_mass[b] = R; a.flags[b] = f;
+                    s_token = pick;
+                }
+            } else if (last >= 0) {
+                // rounding: the target lies beyond the tile's last edge
+                if (lane == 0) {
+                    a.out_token[b] = last; a.resid_mass[b] = R; a.flags[b] = flags | OD_SF_BOUNDARY;
+                    s_token = last;
+                }
+            }                                       // else: the tile holds no mass after all
         }
-        if (attempt == 1) {
-            if (threadIdx.x == 0) s_tile = -1;
-            __syncthreads();
-            break;
-        }
-        // no residual mass: draw from p_j instead (rare; this block redoes the row)
+        __syncthreads();
+        if (s_token >= 0) return;
+        if (!residual || attempt == 1) break;
+        // no usable residual mass: draw from p_j instead (rare; this block redoes the row)
         residual = false;
         flags |= OD_SF_ZERO_MASS;
-        for (int t_lo = warp * 2; t_lo < ntiles; t_lo += WARPS * 2)
-            warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 2 < ntiles ? t_lo + 2 : ntiles, lane, sums);
+        for (int t_lo = warp * 4; t_lo < ntiles; t_lo += WARPS * 4)
+            warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 4 < ntiles ? t_lo + 4 : ntiles, lane, tile_val);
+        __syncthreads();
+        for (int t = threadIdx.x; t < ntiles; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, tile_val[t]);
         __syncthreads();
     }
-    if (s_tile < 0 || s_tile == 0x7FFFFFFF) {       // no mass at all (non-finite input)
-        if (threadIdx.x == 0) {
-            a.out_token[b] = -1; a.resid_mass[b] = (float)(s_total / (double)q.S);
-            a.flags[b] = flags | OD_SF_ZERO_MASS;
-            a.ticket[b] = 0;
-        }
-        return;
-    }
-    if (warp != 0) return;
-
-    // ---- warp 0 scans inside the chosen tile ----
-    const int tile = s_tile;
-    const double Rn = s_total;                      // unnormalised total
-    float r[EPT];
-    tile_values<DTYPE>(q, a, residual, tile, lane, r);
-    const double mine = lane_sum(r);
-    double incl = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const double v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-        if (lane >= off) incl += v;
-    }
-    const double base = s_before + (incl - mine);   // sum before this lane's first id
-    const int t0 = tile * OD_SAMPLE_TILE + lane * EPT;
-    int my_pick = 0x7FFFFFFF, my_last = -1;
-    double lo = 0.0, hi = 0.0;
-    float run = 0.f;                                // same fp32 order as lane_sum
-    double c = base;
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-        run = e == 0 ? r[0] : run + r[e];
-        const double nc = base + (double)run;
-        if (r[e] > 0.f) my_last = t0 + e;
-        if (my_pick == 0x7FFFFFFF && nc > target) { my_pick = t0 + e; lo = c; hi = nc; }
-        c = nc;
-    }
-    int pick = my_pick, last = my_last;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        pick = min(pick, __shfl_xor_sync(0xFFFFFFFFu, pick, off));
-        last = max(last, __shfl_xor_sync(0xFFFFFFFFu, last, off));
-    }
-    const float R = (float)(Rn / (double)q.S);      // residual mass (1 for the free token)
-    if (pick != 0x7FFFFFFF) {
-        if (my_pick == pick) {                      // exactly one lane owns the picked id
-            const double margin = fmin(target - lo, hi - target);
-            if (margin <= OD_TAU_SAMPLE * Rn) flags |= OD_SF_BOUNDARY;
-            a.out_token[b] = pick;
-            a.resid_mass[b] = R;
-            a.flags[b] = flags;
-            a.ticket[b] = 0;
-        }
-    } else if (lane == 0) {
-        // rounding: target beyond the tile's last edge
-        a.out_token[b] = last;
-        a.resid_mass[b] = R;
-        a.flags[b] = flags | OD_SF_BOUNDARY | (last < 0 ? OD_SF_ZERO_MASS : 0u);
-        a.ticket[b] = 0;
+    if (threadIdx.x == 0) {                         // no mass at all (non-finite input)
+        a.out_token[b] = -1; a.resid_mass[b] = (float)(s_total / (double)q.S);
+        a.flags[b] = flags | OD_SF_ZERO_MASS;
     }
 }
 
@@ -406,13 +552,15 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
     a.n_accepted = n_accepted; a.temperature = temperature; a.seed = seed; a.step = step;
     a.vocab_map = c->d_vocab_map; a.inv_map = c->d_inv_map;
     a.out_token = out_token; a.resid_mass = resid_mass; a.flags = flags;
-    a.tile_sums = c->d_tile_sums; a.ticket = c->d_samp_ticket;
+    a.tile_val = c->d_tile_sums; a.ticket = c->d_samp_ticket;
+    a.mapped_t = c->d_mapped_t; a.mapped_d = c->d_mapped_d; a.list_width = c->list_width;
     c->info[2] = (int64_t)blocks_x * B;
     c->info[3] = tpw;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks_x, (unsigned)B);
     cfg.blockDim = dim3(OD_SAMPLE_THREADS);
+    cfg.dynamicSmemBytes = (size_t)ntiles * 8;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -106,37 +106,6 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
     return d;
 }
 
-// Packed fp32 pairs (one instruction for two lanes of arithmetic on sm_100).
-__device__ __forceinline__ uint64_t f2_pack(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void f2_unpack(uint64_t v, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-// acc += (exp2(lo*scale - c), exp2(hi*scale - c))
-__device__ __forceinline__ uint64_t f2_exp_acc(uint64_t acc, float lo, float hi, uint64_t scale2, uint64_t nc2)
-{
-    float e0, e1;
-    f2_unpack(f2_fma(f2_pack(lo, hi), scale2, nc2), e0, e1);
-    return f2_add(acc, f2_pack(od_ex2(e0), od_ex2(e1)));
-}
-
 // Running state of one thread inside a segment.
 template <int DTYPE>
 struct Lane {
