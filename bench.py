@@ -53,7 +53,7 @@ def parse():
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--pool", type=int, default=0, help="distinct step buffers (0 = enough for 4x L2)")
     ap.add_argument("--e2e-steps", type=int, default=8)
-    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
@@ -127,13 +127,23 @@ def measured_peak():
 
 
 def ncu_traffic(workload: str):
-    """Per-launch DRAM bytes of od_verify from the committed ncu summary, if any."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
+    """Per-launch DRAM bytes (read + write) of the stream kernel from the committed ncu
+    summary profiles/traffic.txt, or None when there is no figure for this workload or
+    the kernel source has changed since the counters were taken. Line format:
+    <workload> <bytes per launch> <sha256 of od_verify.cu at capture time>."""
+    import hashlib
     try:
-        with open(p) as f:
-            return json.load(f).get(workload)
+        src = os.path.join(ROOT, "paper_2507_02659_b200", "csrc", "od_verify.cu")
+        with open(src, "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+        with open(os.path.join(ROOT, "profiles", "traffic.txt")) as f:
+            for line in f:
+                t = line.split()
+                if len(t) >= 3 and not line.startswith("#") and t[0] == workload and t[2] == digest:
+                    return float(t[1])
     except Exception:
-        return None
+        pass
+    return None
 
 
 def step_bytes(s):
@@ -141,26 +151,26 @@ def step_bytes(s):
     return sum(x.numel() * x.element_size() for x in t)
 
 
-def oracle_time(w, st, steps, seconds):
-    """Oracle on host cores, one full batch per step, until `seconds` have passed
-    (at least one step). Returns (tokens, elapsed_s, steps_done, threads)."""
+def oracle_time(w, st, host_steps, seconds):
+    """Oracle on host cores over `host_steps` (CPU StepInputs, cycled), one full batch
+    per step, until `seconds` have passed. Returns (tokens, elapsed_s, steps_done, threads)."""
     import oracle
-    from paper_2507_02659_b200 import synth
     cache = oracle.Cache(st.runs, st.run_len, st.run_target)
     threads = oracle.max_threads()
-    tokens, elapsed, done = 0, 0.0, 0
-    for i in range(steps):
-        s = synth.make_step(w, st, i, device="cpu")
+    prepared = []
+    for s in host_steps:
         lg, code = oracle.logits_to_numpy(s.logits)
-        args = (cache, st.vocab_map, w.v_p, s.draft_ids.numpy(), s.draft_len.numpy(), s.q_sel.numpy(),
-                s.q_rows.numpy(), lg, code, s.temperature.numpy(), s.seed.numpy().astype(np.uint64), i)
+        prepared.append((s, (cache, st.vocab_map, w.v_p, s.draft_ids.numpy(), s.draft_len.numpy(),
+                             s.q_sel.numpy(), s.q_rows.numpy(), lg, code, s.temperature.numpy(),
+                             s.seed.numpy().astype(np.uint64))))
+    tokens, elapsed, done = 0, 0.0, 0
+    while elapsed < seconds:
+        s, args = prepared[done % len(prepared)]
         t0 = time.perf_counter()
-        oracle.step_batch(*args, threads=threads)
+        oracle.step_batch(*args, done, threads=threads)
         elapsed += time.perf_counter() - t0
         tokens += int(s.draft_len.sum())
         done += 1
-        if elapsed >= seconds:
-            break
     return tokens, elapsed, done, threads
 
 
@@ -387,9 +397,11 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not a.no_cpu_baseline:
         nseq = min(w.B, 64)
-        tok, el, done, threads = oracle_time(synth.scaled(w, B=nseq), st, 64, a.cpu_seconds)
+        host_steps = [pool[i].slice(0, nseq).to("cpu") for i in range(min(P, 3))]
+        tok, el, done, threads = oracle_time(w, st, host_steps, a.cpu_seconds)
         cpu = {"value": tok / el, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": f"{done} steps of {nseq} of the batch's {w.B} sequences ({el:.1f} s of oracle time)"}
+               "sample": f"{done} steps of {nseq} of the batch's {w.B} sequences, cycling {len(host_steps)} "
+                         f"distinct steps ({el:.1f} s of oracle time)"}
 
     if rank == 0:
         acc = sum(int(vos[i].n_accepted.sum().item()) for i in range(P))
@@ -405,12 +417,12 @@ def main():
                                     f"{P * logit_bytes / 2**20:.0f} MiB of logits cycled",
                        "launch": "K steps captured in one CUDA graph" if not a.no_graph else "eager launches",
                        "parallelism": f"batch sharding x{world}, no collective"},
-            "gpu_launches": 3 * a.steps,
+            "gpu_launches": 4 * a.steps,
             "kernels_ms_per_step": {"od_map_proposals": ms_k1 / a.steps, "od_verify": ms_k2 / a.steps,
                                     "od_sample_residual": ms_k3 / a.steps,
                                     "step_repeats": len(extra),
                                     "step_repeat_median_ms": (statistics.median(extra) / a.steps) if extra else None},
-            "roofline": {"kernel": "od_verify", "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": "od_verify (od_verify_stream_kernel + od_verify_decide_kernel)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                          "bytes_per_launch": k2_bytes_per_launch,
                          "us_per_launch": 1e3 * k2_ms_per_launch,
