@@ -95,6 +95,7 @@ enum od_counter {
  * arithmetic only inside these margins; such decisions are flagged. */
 #define OD_TAU_ACCEPT 1.0e-5f
 #define OD_TAU_SAMPLE 2.0e-6
+#define OD_TAU_EXIT 4.0e-6f
 
 #define OD_MAX_K 16      /* largest K_max */
 #define OD_NOALLOC_MAX_ROWS 1024 /* od_verify_noalloc: largest B * (K_max + 1) */
@@ -220,6 +221,26 @@ int32_t od_sample_residual(od_ctx *ctx, int32_t B, int32_t K_max,
                            const uint64_t *seed, uint64_t step,
                            int32_t *out_token, float *resid_mass,
                            uint32_t *sample_flags, void *stream);
+
+/* Adaptive drafting, exit rule (Section 3.3, Eq. (4)-(6)). From the acceptance
+ * head's outputs f_phi(e_i) of the proposed tokens:
+ *   reject_prob[b,k] = 1 - prod_{i<=k} sigmoid(head_logits[b,i])   (some token up
+ *   to k is rejected), and draft_len[b] = the first k (1-based) at which that
+ *   probability exceeds gamma, or avail_len[b] if it never does. The token whose
+ *   test fires is part of the proposal. The head network itself is not part of
+ *   this library.
+ *   in  (device) head_logits float[B,K_max]; avail_len int32[B] tokens the drafter
+ *                has produced per sequence, clamped to [0, K_max] (NULL = K_max);
+ *                gamma in [0, 1] (INVALID_ARG otherwise)
+ *   out (device) draft_len int32[B] (what od_map_proposals takes);
+ *                reject_prob float[B,K_max], 0 at and beyond avail_len (may be NULL);
+ *                exit_flags uint32[B], bit k: |reject_prob - gamma| <= OD_TAU_EXIT
+ *                at a token up to the exit, where fp32 may decide differently
+ *                from exact arithmetic (may be NULL).
+ * Asynchronous on `stream`; allocates nothing. */
+int32_t od_exit_rule(od_ctx *ctx, int32_t B, int32_t K_max, const float *head_logits,
+                     const int32_t *avail_len, float gamma, int32_t *draft_len,
+                     float *reject_prob, uint32_t *exit_flags, void *stream);
 
 /* Step 2 without any allocation (the paper has no counterpart: this entry
  * point exists for the way some programs are built, not for the method).

@@ -24,13 +24,13 @@ OD_CNT_CACHE_HITS, OD_CNT_UNMAPPED_STOPS, OD_CNT_INVALID_IDS, OD_CNT_MAPPED_TOKE
 OD_CNT_COUNT = 4
 OD_VF_BOUNDARY_MASK, OD_VF_BAD_TEMPERATURE, OD_VF_NONFINITE = 0xFFFF, 0x10000, 0x20000
 OD_SF_BOUNDARY, OD_SF_ZERO_MASS, OD_SF_BAD_TEMPERATURE, OD_SF_BONUS = 0x1, 0x2, 0x4, 0x10
-OD_TAU_ACCEPT, OD_TAU_SAMPLE = 1.0e-5, 2.0e-6
+OD_TAU_ACCEPT, OD_TAU_SAMPLE, OD_TAU_EXIT = 1.0e-5, 2.0e-6, 4.0e-6
 OD_MAX_K = 16
 OD_NOALLOC_MAX_ROWS = 1024
 
 EXPORTS = ["od_create", "od_destroy", "od_set_vocab_map", "od_cache_build", "od_set_option",
            "od_map_proposals", "od_verify", "od_sample_residual", "od_host_step_reserve",
-           "od_step_host", "od_verify_noalloc", "od_last_launch_info", "od_status_string", "od_version"]
+           "od_step_host", "od_verify_noalloc", "od_exit_rule", "od_last_launch_info", "od_status_string", "od_version"]
 
 
 class OdError(RuntimeError):
@@ -63,6 +63,7 @@ def lib():
         L.od_sample_residual.argtypes = ([vp, i32, i32, vp, i32, i64, i64] + [vp] * 13 + [u64]
                                          + [vp] * 3 + [vp])
         L.od_verify_noalloc.argtypes = [i32, i32, i32, vp, i32, i64, i64] + [vp] * 6 + [u64] + [vp] * 7 + [vp]
+        L.od_exit_rule.argtypes = [vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp]
         L.od_host_step_reserve.argtypes = [vp, i32]
         L.od_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp, u64] + [vp] * 7 + [vp]
         L.od_last_launch_info.argtypes = [vp, i32]
@@ -269,6 +270,19 @@ def od_verify_noalloc(target_vocab: int, logits, mp: MapOut, temperature, seed, 
         _dp(out.ratio, f32, d), _dp(out.n_accepted, i32, d), _dp(out.n_draft_accepted, i32, d),
         _dp(out.flags, i32, d), _stream(d)), "od_verify_noalloc")
     return out
+
+
+def od_exit_rule(ctx: Context, head_logits, avail_len, gamma: float):
+    """Eq. (4)-(6): (draft_len int32 [B], reject_prob f32 [B, K], exit_flags int32 [B])."""
+    B, K = head_logits.shape
+    d, i32, f32 = ctx.device, torch.int32, torch.float32
+    draft_len = torch.zeros(B, dtype=i32, device=d)
+    reject = torch.zeros(B, K, dtype=f32, device=d)
+    flags = torch.zeros(B, dtype=i32, device=d)
+    _check(lib().od_exit_rule(ctx.handle, B, K, _dp(head_logits, f32, d), _dp(avail_len, i32, d),
+                              C.c_float(gamma), _dp(draft_len, i32, d), _dp(reject, f32, d),
+                              _dp(flags, i32, d), _stream(d)), "od_exit_rule")
+    return draft_len, reject, flags
 
 
 def od_sample_residual(ctx: Context, logits, vo: VerifyOut, q_rows, draft_ids, mp: MapOut,

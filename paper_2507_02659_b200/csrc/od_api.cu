@@ -321,6 +321,20 @@ int32_t od_sample_residual(od_ctx *c, int32_t B, int32_t K_max, const void *logi
     return OD_OK;
 }
 
+int32_t od_exit_rule(od_ctx *c, int32_t B, int32_t K_max, const float *head_logits,
+                     const int32_t *avail_len, float gamma, int32_t *draft_len, float *reject_prob,
+                     uint32_t *exit_flags, void *stream)
+{
+    if (!c || B < 0 || K_max < 1 || K_max > OD_MAX_K) return OD_ERR_INVALID_ARG;
+    if (!head_logits || !draft_len) return OD_ERR_INVALID_ARG;
+    if (!(gamma >= 0.f && gamma <= 1.f)) return OD_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    OD_CUDA(od_launch_exit(B, K_max, head_logits, avail_len, gamma, draft_len, reject_prob, exit_flags,
+                           (cudaStream_t)stream));
+    return OD_OK;
+}
+
 int32_t od_host_step_reserve(od_ctx *c, int32_t logit_dtype)
 {
     if (!c) return OD_ERR_INVALID_ARG;

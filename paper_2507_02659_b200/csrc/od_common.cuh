@@ -92,6 +92,10 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
                              cudaStream_t s);
 
+cudaError_t od_launch_exit(int32_t B, int32_t K_max, const float *head_logits, const int32_t *avail_len,
+                           float gamma, int32_t *draft_len, float *reject_prob, uint32_t *flags,
+                           cudaStream_t s);
+
 // 64-bit key of a run of draft ids: (id + 1) in 16 bits per position, first id
 // in the low bits. Never 0 for a non-empty run.
 __host__ __device__ inline uint64_t od_pack_run(const int32_t *ids, int len)

@@ -334,3 +334,33 @@ def test_host_step_matches_device_step(cuda_device):
     assert torch.equal(out.verify_flags, vo.flags.cpu())
     assert torch.equal(out.sample_flags, so.flags.cpu())
     ctx.close()
+
+
+# ------------------------------------------------------------ adaptive drafting, exit rule
+@pytest.mark.parametrize("gamma", [0.3, 0.7])
+def test_exit_rule_matches_the_oracle(cuda_device, gamma):
+    """Eq. (4)-(6): lengths equal the fp64 oracle's except where the kernel flagged a
+    decision within its margin; probabilities within fp32 rounding."""
+    from oracle import exit_rule as er
+    rng = np.random.default_rng(11)
+    B, K = 3000, 10
+    f = rng.normal(2.0, 1.5, size=(B, K)).astype(np.float32)
+    f[:50] = 40.0                                  # never exits
+    f[50:100] = -40.0                              # exits at the first token
+    avail = rng.integers(0, K + 1, size=B).astype(np.int32)
+    ctx = od.Context(cuda_device, 100, 100, 4, K)
+    length, reject, flags = od.od_exit_rule(ctx, torch.from_numpy(f).to(cuda_device),
+                                            torch.from_numpy(avail).to(cuda_device), gamma)
+    torch.cuda.synchronize()
+    want_len, want_rej = er.exit_rule(f, avail, gamma)
+    length, reject, flags = length.cpu().numpy(), reject.cpu().numpy(), flags.cpu().numpy()
+    np.testing.assert_allclose(reject, want_rej, rtol=0, atol=3e-6)
+    differ = length != want_len
+    assert (flags[differ] != 0).all(), "a length that differs from the oracle's must be flagged"
+    assert differ.sum() <= 3 and (flags != 0).sum() <= 10
+    assert (length[avail == 0] == 0).all() and (length <= avail).all()
+    # the result feeds od_map_proposals as draft_len: same dtype and shape
+    assert length.dtype == np.int32 and length.shape == (B,)
+    with pytest.raises(od.OdError):
+        od.od_exit_rule(ctx, torch.zeros(2, K, device=cuda_device), None, 1.5)
+    ctx.close()
