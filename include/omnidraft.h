@@ -133,6 +133,52 @@ int32_t od_cache_build(od_ctx *ctx, const int32_t *host_runs,
                        const int32_t *host_len, const int32_t *host_target,
                        int64_t E);
 
+/* ---- online cache -------------------------------------------------------- */
+
+/* The cache as Algorithm 1 grows it (cache-update line: an n-gram that is not in
+ * the cache yet is added) and bounds it (App. D.5: a maximum size with LRU, which
+ * evicts the n-gram not accessed for the longest time, or LFU, which evicts the one
+ * with the lowest access frequency). Where the paper is silent: an access is a
+ * cached run that od_map_proposals actually merges (and the insertion itself); time
+ * is a clock the caller sets, one tick per verification step; eviction is an explicit
+ * trim; ties go by the run's packed key; entries inserted at the current clock are
+ * evicted last.
+ *
+ * od_cache_configure installs an EMPTY online cache for at most `max_entries`
+ * entries after a trim (policy 0 = LRU, 1 = LFU) and batches of at most `max_insert`
+ * candidates; it replaces any earlier cache (od_cache_build does the reverse) and is
+ * synchronous. Needs draft_vocab <= 65535 (UNSUPPORTED otherwise). */
+int32_t od_cache_configure(od_ctx *ctx, int64_t max_entries, int32_t policy,
+                           int32_t max_insert);
+
+/* The clock that stamps accesses (od_map_proposals) and insertions enqueued from
+ * now on. Host-side; STATE without an online cache. */
+int32_t od_cache_set_clock(od_ctx *ctx, uint32_t clock);
+
+/* Adds the candidates that are not in the cache yet. device: runs int32[N,4]
+ * (draft ids, the first len[i] are used), len int32[N] in 2..4, target int32[N].
+ * Of several candidates with the same run the one with the lowest index wins, as
+ * if they were added one after the other; malformed candidates (length, ids or
+ * target out of range) are skipped. New entries get the current clock as time of
+ * insertion and of last access, and frequency 1. Asynchronous on `stream`; must be
+ * ordered with od_map_proposals on the same context. N <= max_insert. */
+int32_t od_cache_insert(od_ctx *ctx, int32_t N, const int32_t *runs,
+                        const int32_t *len, const int32_t *target, void *stream);
+
+/* If the cache holds k > 0 entries more than max_entries, drops the k entries that
+ * come first in the order (inserted at the current clock? no before yes; then last
+ * access clock for LRU or frequency for LFU, ascending; then the run's packed key,
+ * ascending) and rebuilds the table. Asynchronous on `stream` (a fixed sequence of
+ * small kernels, no host round trip); calls enqueued afterwards see the new table. */
+int32_t od_cache_trim(od_ctx *ctx, void *stream);
+
+/* Contents of the online cache, for inspection and tests: synchronises the device,
+ * writes up to max_out entries (host arrays: runs int32[max_out,4] padded with -1,
+ * len, target, and, if not NULL, the last-access clock and the frequency) in no
+ * particular order, and the total number of entries to *n_out. */
+int32_t od_cache_dump(od_ctx *ctx, int64_t max_out, int32_t *runs, int32_t *len,
+                      int32_t *target, uint32_t *stamp, uint32_t *freq, int64_t *n_out);
+
 /* Tuning knobs, mainly for experiments. Names: "verify_blocks_per_sm" (thread
  * blocks of od_verify per multiprocessor, 1..8, 0 = automatic),
  * "sample_tiles_per_warp" (256-id tiles one warp of od_sample_residual sums,

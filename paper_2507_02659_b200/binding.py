@@ -30,7 +30,8 @@ OD_NOALLOC_MAX_ROWS = 1024
 
 EXPORTS = ["od_create", "od_destroy", "od_set_vocab_map", "od_cache_build", "od_set_option",
            "od_map_proposals", "od_verify", "od_sample_residual", "od_host_step_reserve",
-           "od_step_host", "od_verify_noalloc", "od_exit_rule", "od_last_launch_info", "od_status_string", "od_version"]
+           "od_step_host", "od_verify_noalloc", "od_exit_rule", "od_cache_configure", "od_cache_set_clock",
+           "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_last_launch_info", "od_status_string", "od_version"]
 
 
 class OdError(RuntimeError):
@@ -64,6 +65,11 @@ def lib():
                                          + [vp] * 3 + [vp])
         L.od_verify_noalloc.argtypes = [i32, i32, i32, vp, i32, i64, i64] + [vp] * 6 + [u64] + [vp] * 7 + [vp]
         L.od_exit_rule.argtypes = [vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp]
+        L.od_cache_configure.argtypes = [vp, i64, i32, i32]
+        L.od_cache_set_clock.argtypes = [vp, C.c_uint32]
+        L.od_cache_insert.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.od_cache_trim.argtypes = [vp, vp]
+        L.od_cache_dump.argtypes = [vp, i64, vp, vp, vp, vp, vp, C.POINTER(i64)]
         L.od_host_step_reserve.argtypes = [vp, i32]
         L.od_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp, u64] + [vp] * 7 + [vp]
         L.od_last_launch_info.argtypes = [vp, i32]
@@ -152,6 +158,36 @@ class Context:
             raise ValueError("cache arrays disagree on the number of entries")
         _check(lib().od_cache_build(self.handle, _hp(runs), _hp(run_len), _hp(run_target), E),
                "od_cache_build")
+
+    # ---- online cache (insertion of unseen n-grams, LRU / LFU trim)
+    def cache_configure(self, max_entries: int, policy: int, max_insert: int):
+        _check(lib().od_cache_configure(self.handle, int(max_entries), int(policy), int(max_insert)),
+               "od_cache_configure")
+
+    def cache_set_clock(self, clock: int):
+        _check(lib().od_cache_set_clock(self.handle, int(clock) & 0xFFFFFFFF), "od_cache_set_clock")
+
+    def cache_insert(self, runs: torch.Tensor, run_len: torch.Tensor, run_target: torch.Tensor):
+        d, i32 = self.device, torch.int32
+        N = int(run_len.shape[0])
+        if tuple(runs.shape) != (N, 4) or run_target.shape[0] != N:
+            raise ValueError("candidates must be runs [N, 4], len [N], target [N]")
+        _check(lib().od_cache_insert(self.handle, N, _dp(runs, i32, d), _dp(run_len, i32, d),
+                                     _dp(run_target, i32, d), _stream(d)), "od_cache_insert")
+
+    def cache_trim(self):
+        _check(lib().od_cache_trim(self.handle, _stream(self.device)), "od_cache_trim")
+
+    def cache_dump(self):
+        """{run tuple: (target, last-access clock, frequency)} of the online cache (synchronous)."""
+        n = C.c_int64(0)
+        _check(lib().od_cache_dump(self.handle, 0, None, None, None, None, None, C.byref(n)), "od_cache_dump")
+        E = n.value
+        runs = np.full((max(E, 1), 4), -1, np.int32); ln = np.zeros(max(E, 1), np.int32)
+        tg = np.zeros(max(E, 1), np.int32); st = np.zeros(max(E, 1), np.uint32); fr = np.zeros(max(E, 1), np.uint32)
+        _check(lib().od_cache_dump(self.handle, E, _hp(runs), _hp(ln), _hp(tg), _hp(st), _hp(fr), C.byref(n)),
+               "od_cache_dump")
+        return {tuple(int(x) for x in runs[i, :ln[i]]): (int(tg[i]), int(st[i]), int(fr[i])) for i in range(E)}
 
     def set_option(self, name: str, value: int):
         _check(lib().od_set_option(self.handle, name.encode(), int(value)), "od_set_option")

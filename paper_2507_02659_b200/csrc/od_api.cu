@@ -44,6 +44,7 @@ int32_t dev_alloc(T **p, size_t n)
 
 void free_all(od_ctx *c)
 {
+    od_cache_free_dynamic(c);
     void *ptrs[] = {c->d_vocab_map, c->d_inv_map, c->d_mapped_t, c->d_mapped_d, c->d_keys, c->d_vals, c->d_partials,
                     c->d_tile_sums,
                     c->d_samp_ticket, c->s_logits, c->s_q_rows, c->s_q_sel, c->s_temperature,
@@ -230,6 +231,7 @@ int32_t od_cache_build(od_ctx *c, const int32_t *host_runs, const int32_t *host_
         }
     }
     OD_CUDA(cudaDeviceSynchronize());
+    od_cache_free_dynamic(c);                               // a static cache replaces an online one
     if (c->d_keys) { cudaFree(c->d_keys); c->d_keys = nullptr; }
     if (c->d_vals) { cudaFree(c->d_vals); c->d_vals = nullptr; }
     c->cap = 0;

@@ -36,6 +36,20 @@ struct od_ctx {
     int32_t *d_vals;                // [cap]
     int64_t cap;                    // power of two, multiple of 32, or 0
 
+    // online cache (od_cache_configure): per-slot access data of the current table, a
+    // second table that od_cache_trim rebuilds into, and the scratch of insert and trim
+    bool dyn;
+    int32_t dyn_policy;             // 0 = LRU, 1 = LFU
+    int64_t dyn_max;                // entries kept by a trim
+    int32_t dyn_max_insert;         // largest batch of od_cache_insert
+    uint32_t clock;                 // stamp of accesses and insertions
+    uint32_t *d_stamp, *d_freq, *d_born;            // [cap]
+    uint64_t *d_keys2; int32_t *d_vals2;            // [cap] spare table
+    uint32_t *d_stamp2, *d_freq2, *d_born2;
+    uint32_t *d_owner;              // [cap] first-wins claims of a batch (0xFFFFFFFF = none)
+    int32_t *d_cand_slot;           // [dyn_max_insert]
+    void *d_trim;                   // trim / size state (device)
+
     // od_verify scratch
     float4 *d_partials;             // [rows][OD_VERIFY_SEG_MAX] (c, sum, max, -), rows of one launch
 
@@ -91,6 +105,8 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              const float *temperature, const uint64_t *seed, uint64_t step,
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
                              cudaStream_t s);
+
+void od_cache_free_dynamic(od_ctx *c);   // frees what od_cache_configure allocated beyond keys / vals
 
 cudaError_t od_launch_exit(int32_t B, int32_t K_max, const float *head_logits, const int32_t *avail_len,
                            float gamma, int32_t *draft_len, float *reject_prob, uint32_t *flags,

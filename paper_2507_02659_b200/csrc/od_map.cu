@@ -14,8 +14,8 @@
 
 namespace {
 
+// returns the slot that holds `key`, or -1
 __device__ __forceinline__ int32_t probe_continue(const uint64_t *__restrict__ keys,
-                                                  const int32_t *__restrict__ vals,
                                                   uint64_t ngroups, uint64_t key, uint64_t g,
                                                   uint64_t k_lane, int lane)
 {
@@ -23,7 +23,7 @@ __device__ __forceinline__ int32_t probe_continue(const uint64_t *__restrict__ k
     // walks at most ngroups groups, so it ends on any table contents
     for (uint64_t step = 0; step < ngroups; ++step) {
         unsigned match = __ballot_sync(0xFFFFFFFFu, k_lane == key);
-        if (match) return __ldg(vals + g * OD_GROUP + (__ffs(match) - 1));
+        if (match) return (int32_t)(g * OD_GROUP + (__ffs(match) - 1));
         unsigned empty = __ballot_sync(0xFFFFFFFFu, k_lane == 0ULL);
         if (empty) return -1;
         g = (g + 1) & (ngroups - 1);
@@ -39,10 +39,12 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
               const int32_t *__restrict__ vals, int64_t cap, int32_t *__restrict__ tgt_ids,
               float *__restrict__ q_prime, int32_t *__restrict__ span_start,
               int32_t *__restrict__ span_len, int32_t *__restrict__ m_out,
-              uint8_t *__restrict__ tail_kind, uint32_t *__restrict__ counters)
+              uint8_t *__restrict__ tail_kind, uint32_t *__restrict__ counters,
+              uint32_t *__restrict__ stamp, uint32_t *__restrict__ freq, uint32_t clock)
 {
     __shared__ int32_t s_ids[OD_MAX_K];
     __shared__ int32_t s_hit[OD_MAX_K][OD_NGRAM_MAX + 1];   // [offset][length] -> target or -1
+    __shared__ int32_t s_slot[OD_MAX_K][OD_NGRAM_MAX + 1];  // the table slot of that hit
     __shared__ int32_t s_direct[OD_MAX_K];                  // direct map of the id at each offset, or -1
     __shared__ float s_q[OD_MAX_K];                         // q(d) of each offset
 
@@ -69,6 +71,7 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
             s_q[s] = q_sel[(size_t)b * K_max + s];
         }
         int32_t hit[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
+        int32_t slot[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
         if (cap > 0) {
             const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
             uint64_t key[OD_NGRAM_MAX + 1], grp[OD_NGRAM_MAX + 1], kl[OD_NGRAM_MAX + 1];
@@ -90,11 +93,15 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
                 kl[L] = valid[L] ? __ldg(keys + grp[L] * OD_GROUP + lane) : 0ULL;
 #pragma unroll
             for (int L = 2; L <= OD_NGRAM_MAX; ++L)
-                if (valid[L]) hit[L] = probe_continue(keys, vals, ngroups, key[L], grp[L], kl[L], lane);
+                if (valid[L]) {
+                    slot[L] = probe_continue(keys, ngroups, key[L], grp[L], kl[L], lane);
+                    // an entry whose value is not set yet does not exist (a concurrent batch insert writes it last)
+                    if (slot[L] >= 0) hit[L] = __ldg(vals + slot[L]);
+                }
         }
         if (lane == 0) {
 #pragma unroll
-            for (int L = 2; L <= OD_NGRAM_MAX; ++L) s_hit[s][L] = hit[L];
+            for (int L = 2; L <= OD_NGRAM_MAX; ++L) { s_hit[s][L] = hit[L]; s_slot[s][L] = slot[L]; }
         }
     }
     __syncthreads();
@@ -114,6 +121,10 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
                 for (int j = 1; j < L; ++j) prod *= s_q[pos + j];
                 tgt_ids[o + m] = t; q_prime[o + m] = prod;
                 span_start[o + m] = pos; span_len[o + m] = L;
+                if (stamp) {                                // an access: recency and frequency of the entry
+                    atomicMax(stamp + s_slot[pos][L], clock);
+                    atomicAdd(freq + s_slot[pos][L], 1u);
+                }
                 ++m; pos += L; ++hits;
                 continue;
             }
@@ -162,5 +173,6 @@ cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *dr
     return cudaLaunchKernelEx(&cfg, od_map_kernel, B, K_max, c->v_q, draft_ids, draft_len, q_sel,
                               (const int32_t *)c->d_vocab_map, (const uint64_t *)c->d_keys,
                               (const int32_t *)c->d_vals, c->cap, tgt_ids, q_prime, span_start,
-                              span_len, m, tail_kind, counters);
+                              span_len, m, tail_kind, counters, c->dyn ? c->d_stamp : (uint32_t *)nullptr,
+                              c->dyn ? c->d_freq : (uint32_t *)nullptr, c->clock);
 }
