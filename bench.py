@@ -59,6 +59,8 @@ def parse():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--cache-update", action="store_true",
                     help="time the online-cache update path (insert + trim) instead of the verification step")
+    ap.add_argument("--distill", action="store_true",
+                    help="time the distillation loss + gradient (Eq. 3) of the step's proposals instead")
     ap.add_argument("--verify-blocks-per-sm", type=int, default=0)
     ap.add_argument("--verify-waves", type=int, default=0)
     ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
@@ -269,10 +271,63 @@ def run_cache_update(a):
     ctx.close()
 
 
+def run_distill(a):
+    """od_distill_loss on the bench workload's proposals (after od_map_proposals and
+    od_verify, which are not timed): draft positions/s and the HBM rate of the drafter
+    rows read and gradient rows written."""
+    from paper_2507_02659_b200 import binding as od
+    from paper_2507_02659_b200 import synth
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    w = synth.paper_config(a.config)
+    st = synth.make_static(w)
+    ctx = od.Context(dev, w.v_q, w.v_p, w.B, w.k_max)
+    ctx.set_vocab_map(st.vocab_map)
+    ctx.cache_build(st.runs, st.run_len, st.run_target)
+    P = 6
+    B, K = w.B, w.k_max
+    pool = [synth.make_step(w, st, i, device=dev) for i in range(P)]
+    mps = [od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel) for s in pool]
+    vos = [od.od_verify(ctx, s.logits, mps[i], s.temperature, s.seed, i) for i, s in enumerate(pool)]
+    loss = [torch.zeros(B, K, device=dev) for _ in range(P)]
+    grad = [torch.empty(B, K, w.v_q, device=dev) for _ in range(P)]      # P x 49 MB: larger than L2 together with q
+    def call(i):
+        s = pool[i % P]
+        od.od_distill_loss(ctx, s.q_rows, s.draft_ids, mps[i % P], s.logits, vos[i % P], s.temperature, 0.2, 0,
+                           loss=loss[i % P], grad=grad[i % P])
+    for i in range(max(3, a.warmup)):
+        call(i)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(a.steps):
+            call(i)
+    g.replay(); torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); g.replay(); e1.record(); torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / a.steps
+    active = sum(int(mps[i % P].span_len[torch.arange(K, device=dev)[None, :] < mps[i % P].m[:, None]].sum())
+                 for i in range(a.steps)) / a.steps
+    bytes_per_call = active * 2 * w.v_q * 4 + (B * K - active) * w.v_q * 4
+    peak, peak_src = measured_peak()
+    print(json.dumps({
+        "metric": "distilled_draft_positions_per_sec", "value": active / (ms * 1e-3), "unit": "positions/s",
+        "n_gpus": 1, "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "B": B, "k_max": K, "draft_vocab": w.v_q, "target_vocab": w.v_p,
+                   "l2_policy": f"{P} distinct step buffers (q rows + gradient rows {P * 2 * B * K * w.v_q * 4 / 2**20:.0f} MiB)"},
+        "roofline": {"kernel": "od_distill_kernel", "bound": "hbm", "achieved": bytes_per_call / (ms * 1e-3) / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": bytes_per_call / (ms * 1e-3) / 1e9 / peak,
+                     "peak_source": peak_src, "bytes_per_launch": bytes_per_call, "traffic": None},
+        "active_positions_per_step": active}))
+    ctx.close()
+
+
 def main():
     a = parse()
     if a.impl == "reference":
         return run_reference(a)
+    if a.distill:
+        return run_distill(a)
     if a.cache_update:
         return run_cache_update(a)
     if a.warmup < 3:

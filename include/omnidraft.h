@@ -268,6 +268,33 @@ int32_t od_sample_residual(od_ctx *ctx, int32_t B, int32_t K_max,
                            int32_t *out_token, float *resid_mass,
                            uint32_t *sample_flags, void *stream);
 
+/* Hybrid cross-vocabulary distillation loss (Section 3.2, Eq. (3)) of the proposals
+ * of one verification step, per draft position j, and its gradient with respect to
+ * the drafter's logits z (q = softmax(z)):
+ *   j directly mapped (its piece has one sub-token, target position i):
+ *       loss = KL(q' || p_i) = sum over mapped draft ids d of q(d) (ln q(d) - ln p_i(map[d])),
+ *       grad(d) = q(d) (g(d) - sum_e q(e) g(e)),  g(d) = [d mapped] (ln q(d) - ln p_i(map[d]) + 1);
+ *   j a sub-token of a cached n-gram:  loss = -w ln q(d_j),  grad(d) = w (q(d) - [d == d_j]),
+ *       w = lambda (lambda_mode 0) or the verified target probability p_i(t_i) of the
+ *       n-gram (lambda_mode 1, needs p_sel);
+ *   j not translated (at or after an unmapped stop, beyond K_b) or T_b <= 0: 0.
+ * p_i = softmax(row i / T_b), taken from the logits and from the row statistics that
+ * od_verify wrote (row_max, row_sum). Sums over positions or the batch are the
+ * caller's.
+ *   in  (device) q_rows float[B,K_max,draft_vocab]; draft_ids; tgt_ids, span_start,
+ *                span_len, m from od_map_proposals; logits, strides as for od_verify;
+ *                row_max, row_sum, p_sel from od_verify; temperature float[B]
+ *   out (device) loss float[B,K_max]; grad float[B,K_max,draft_vocab] (may be NULL)
+ * Asynchronous on `stream`; allocates nothing. */
+int32_t od_distill_loss(od_ctx *ctx, int32_t B, int32_t K_max, const float *q_rows,
+                        const int32_t *draft_ids, const int32_t *tgt_ids,
+                        const int32_t *span_start, const int32_t *span_len,
+                        const int32_t *m, const void *logits, int32_t logit_dtype,
+                        int64_t row_stride, int64_t seq_stride, const float *row_max,
+                        const float *row_sum, const float *p_sel,
+                        const float *temperature, float lambda, int32_t lambda_mode,
+                        float *loss, float *grad, void *stream);
+
 /* Adaptive drafting, exit rule (Section 3.3, Eq. (4)-(6)). From the acceptance
  * head's outputs f_phi(e_i) of the proposed tokens:
  *   reject_prob[b,k] = 1 - prod_{i<=k} sigmoid(head_logits[b,i])   (some token up

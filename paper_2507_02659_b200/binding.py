@@ -31,7 +31,7 @@ OD_NOALLOC_MAX_ROWS = 1024
 EXPORTS = ["od_create", "od_destroy", "od_set_vocab_map", "od_cache_build", "od_set_option",
            "od_map_proposals", "od_verify", "od_sample_residual", "od_host_step_reserve",
            "od_step_host", "od_verify_noalloc", "od_exit_rule", "od_cache_configure", "od_cache_set_clock",
-           "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_last_launch_info", "od_status_string", "od_version"]
+           "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_distill_loss", "od_last_launch_info", "od_status_string", "od_version"]
 
 
 class OdError(RuntimeError):
@@ -65,6 +65,8 @@ def lib():
                                          + [vp] * 3 + [vp])
         L.od_verify_noalloc.argtypes = [i32, i32, i32, vp, i32, i64, i64] + [vp] * 6 + [u64] + [vp] * 7 + [vp]
         L.od_exit_rule.argtypes = [vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp]
+        L.od_distill_loss.argtypes = ([vp, i32, i32] + [vp] * 7 + [i32, i64, i64] + [vp] * 4
+                                      + [C.c_float, i32, vp, vp, vp])
         L.od_cache_configure.argtypes = [vp, i64, i32, i32]
         L.od_cache_set_clock.argtypes = [vp, C.c_uint32]
         L.od_cache_insert.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -306,6 +308,25 @@ def od_verify_noalloc(target_vocab: int, logits, mp: MapOut, temperature, seed, 
         _dp(out.ratio, f32, d), _dp(out.n_accepted, i32, d), _dp(out.n_draft_accepted, i32, d),
         _dp(out.flags, i32, d), _stream(d)), "od_verify_noalloc")
     return out
+
+
+def od_distill_loss(ctx: Context, q_rows, draft_ids, mp: MapOut, logits, vo: VerifyOut, temperature,
+                    lam: float, lambda_mode: int = 0, want_grad: bool = True, loss=None, grad=None):
+    """Eq. (3) per draft position: (loss f32 [B, K], grad f32 [B, K, V_q] or None)."""
+    B, K = mp.tgt_ids.shape
+    d, i32, f32 = ctx.device, torch.int32, torch.float32
+    rs, ss = _strides(logits, B, K, ctx.target_vocab)
+    if loss is None:
+        loss = torch.zeros(B, K, dtype=f32, device=d)
+    if grad is None and want_grad:
+        grad = torch.empty(B, K, ctx.draft_vocab, dtype=f32, device=d)
+    _check(lib().od_distill_loss(
+        ctx.handle, B, K, _dp(q_rows, f32, d), _dp(draft_ids, i32, d), _dp(mp.tgt_ids, i32, d),
+        _dp(mp.span_start, i32, d), _dp(mp.span_len, i32, d), _dp(mp.m, i32, d),
+        C.c_void_p(logits.data_ptr()), logit_dtype_code(logits), rs, ss, _dp(vo.row_max, f32, d),
+        _dp(vo.row_sum, f32, d), _dp(vo.p_sel, f32, d), _dp(temperature, f32, d), C.c_float(lam),
+        int(lambda_mode), _dp(loss, f32, d), _dp(grad, f32, d), _stream(d)), "od_distill_loss")
+    return loss, grad
 
 
 def od_exit_rule(ctx: Context, head_logits, avail_len, gamma: float):

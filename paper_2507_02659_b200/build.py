@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libomnidraft.so")
-SOURCES = ["od_api.cu", "od_map.cu", "od_verify.cu", "od_sample.cu", "od_noalloc.cu", "od_exit.cu", "od_cache.cu"]
+SOURCES = ["od_api.cu", "od_map.cu", "od_verify.cu", "od_sample.cu", "od_noalloc.cu", "od_exit.cu", "od_cache.cu", "od_distill.cu"]
 
 
 def _newest_source() -> float:

@@ -323,6 +323,30 @@ int32_t od_sample_residual(od_ctx *c, int32_t B, int32_t K_max, const void *logi
     return OD_OK;
 }
 
+int32_t od_distill_loss(od_ctx *c, int32_t B, int32_t K_max, const float *q_rows,
+                        const int32_t *draft_ids, const int32_t *tgt_ids, const int32_t *span_start,
+                        const int32_t *span_len, const int32_t *m, const void *logits,
+                        int32_t logit_dtype, int64_t row_stride, int64_t seq_stride,
+                        const float *row_max, const float *row_sum, const float *p_sel,
+                        const float *temperature, float lambda, int32_t lambda_mode, float *loss,
+                        float *grad, void *stream)
+{
+    int32_t st = check_step_common(c, B, K_max);
+    if (st != OD_OK) return st;
+    st = check_logits(c, logits, logit_dtype, row_stride, seq_stride, K_max);
+    if (st != OD_OK) return st;
+    if (!q_rows || !draft_ids || !tgt_ids || !span_start || !span_len || !m || !row_max || !row_sum ||
+        !temperature || !loss || (lambda_mode != 0 && lambda_mode != 1) || (lambda_mode == 1 && !p_sel) ||
+        !(lambda >= 0.f))
+        return OD_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    OD_CUDA(od_launch_distill(c, B, K_max, q_rows, draft_ids, tgt_ids, span_start, span_len, m, logits,
+                              logit_dtype, row_stride, seq_stride, row_max, row_sum, p_sel, temperature,
+                              lambda, lambda_mode, loss, grad, (cudaStream_t)stream));
+    return OD_OK;
+}
+
 int32_t od_exit_rule(od_ctx *c, int32_t B, int32_t K_max, const float *head_logits,
                      const int32_t *avail_len, float gamma, int32_t *draft_len, float *reject_prob,
                      uint32_t *exit_flags, void *stream)

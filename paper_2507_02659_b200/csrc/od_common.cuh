@@ -106,6 +106,13 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
                              cudaStream_t s);
 
+cudaError_t od_launch_distill(od_ctx *c, int32_t B, int32_t K_max, const float *q_rows,
+                              const int32_t *draft_ids, const int32_t *tgt_ids, const int32_t *span_start,
+                              const int32_t *span_len, const int32_t *m, const void *logits, int32_t dtype,
+                              int64_t row_stride, int64_t seq_stride, const float *row_max,
+                              const float *row_sum, const float *p_sel, const float *temperature,
+                              float lambda, int32_t lambda_mode, float *loss, float *grad, cudaStream_t s);
+
 void od_cache_free_dynamic(od_ctx *c);   // frees what od_cache_configure allocated beyond keys / vals
 
 cudaError_t od_launch_exit(int32_t B, int32_t K_max, const float *head_logits, const int32_t *avail_len,

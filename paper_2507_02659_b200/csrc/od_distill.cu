@@ -1,0 +1,140 @@
+// Hybrid cross-vocabulary distillation loss (Section 3.2, Eq. (3)) and its gradient
+// with respect to the drafter's logits, per proposed draft position:
+//   directly mapped token (its piece of the translated proposal has one sub-token,
+//   target position i):   L = KL(q' || p_i) = sum over mapped draft ids d of
+//                             q(d) * (ln q(d) - ln p_i(map[d]))
+//   sub-token of a cached n-gram:   L = -lambda * ln q(d_j)   (lambda constant, or the
+//                             verified target probability of the n-gram)
+//   not translated:       L = 0.
+// With q = softmax(z):  KL:  dL/dz(d) = q(d) * (g(d) - sum_e q(e) g(e)),
+//                            g(d) = [d mapped] * (ln q(d) - ln p(map[d]) + 1)
+//                       NLL: dL/dz(d) = lambda * (q(d) - [d == d_j]).
+// ln p_i(t) = (x_t - M_i)/T - ln S_i reuses the row statistics od_verify produced, so
+// the target row is only gathered at the mapped ids, never streamed again.
+//
+// One block of 1024 threads per (sequence, draft position); two sweeps over the draft
+// vocabulary (sums, then gradient; the second sweep finds its inputs in cache), reads
+// coalesced except the one gathered logit per mapped id. Bound by HBM: the drafter's
+// row in, the gradient row out.
+#include <float.h>
+
+#include "od_common.cuh"
+
+namespace {
+
+constexpr int THREADS = 1024;
+
+struct DistillArgs {
+    int32_t B, K_max, v_q, v_p;
+    const float *q_rows;
+    const int32_t *draft_ids, *tgt_ids, *span_start, *span_len, *m;
+    const void *logits;
+    int64_t row_stride, seq_stride;
+    const float *row_max, *row_sum, *p_sel, *temperature;
+    const int32_t *vocab_map;
+    float lambda;
+    int32_t lambda_mode;
+    float *loss, *grad;
+};
+
+__device__ __forceinline__ double block_sum(double v, double *s_red)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) s_red[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int w = 0; w < THREADS / 32; ++w) t += s_red[w];   // the same order in every thread
+    return t;
+}
+
+template <int DTYPE>
+__global__ void __launch_bounds__(THREADS, 2)
+od_distill_kernel(const DistillArgs a)
+{
+    __shared__ double s_red[THREADS / 32];
+    const int b = blockIdx.y, j = blockIdx.x;
+    const int K = a.K_max;
+    int mb = a.m[b];
+    mb = mb < 0 ? 0 : (mb > K ? K : mb);
+    // the piece of the translated proposal that covers draft position j, if any
+    int piece = -1, plen = 0;
+    for (int i = 0; i < mb; ++i) {
+        const int s0 = a.span_start[(size_t)b * K + i], L = a.span_len[(size_t)b * K + i];
+        if (j >= s0 && j < s0 + L) { piece = i; plen = L; }
+    }
+    const float *q = a.q_rows + ((size_t)b * K + j) * a.v_q;
+    float *grad = a.grad ? a.grad + ((size_t)b * K + j) * a.v_q : nullptr;
+    const float T = a.temperature[b];
+    if (piece < 0 || !(T > 0.f)) {                           // not translated: no loss, no gradient
+        if (threadIdx.x == 0) a.loss[(size_t)b * K + j] = 0.f;
+        if (grad)
+            for (int d = threadIdx.x; d < a.v_q; d += THREADS) grad[d] = 0.f;
+        return;
+    }
+    if (plen >= 2) {
+        // ---- a sub-token of a cached n-gram: -w ln q(d_j)
+        const int32_t dj = a.draft_ids[(size_t)b * K + j];
+        const float w = a.lambda_mode == 0 ? a.lambda : a.p_sel[(size_t)b * K + piece];
+        if (threadIdx.x == 0) a.loss[(size_t)b * K + j] = (dj >= 0 && dj < a.v_q) ? -w * logf(q[dj]) : 0.f;
+        if (grad)
+            for (int d = threadIdx.x; d < a.v_q; d += THREADS) grad[d] = w * (__ldg(q + d) - (d == dj ? 1.f : 0.f));
+        return;
+    }
+    // ---- a directly mapped token: KL(q' || p_i) over the mapped ids
+    const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
+    const char *row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)piece * a.row_stride) * esz;
+    const float M = a.row_max[b * (K + 1) + piece];
+    const float ln_S = logf(a.row_sum[b * (K + 1) + piece]);
+    const float inv_T = 1.f / T;
+    // f(d) = ln q(d) - ln p(map[d]) for a mapped d with q(d) > 0, else "no term"
+    auto term = [&](int d, float &qd, float &f) -> bool {
+        const int32_t t = __ldg(a.vocab_map + d);
+        qd = __ldg(q + d);
+        if (t < 0 || !(qd > 0.f)) return false;
+        f = logf(qd) - ((od_load_logit<DTYPE>(row, t) - M) * inv_T - ln_S);
+        return true;
+    };
+    float loss_t = 0.f, qg_t = 0.f;                          // sum q f, sum q (f + 1) over this thread's ids
+#pragma unroll 4
+    for (int d = threadIdx.x; d < a.v_q; d += THREADS) {
+        float qd, f;
+        if (term(d, qd, f)) { loss_t += qd * f; qg_t += qd * (f + 1.f); }
+    }
+    const double loss = block_sum((double)loss_t, s_red);
+    const double qg = block_sum((double)qg_t, s_red);
+    if (threadIdx.x == 0) a.loss[(size_t)b * K + j] = (float)loss;
+    if (grad) {
+        const float gbar = (float)qg;
+#pragma unroll 4
+        for (int d = threadIdx.x; d < a.v_q; d += THREADS) {
+            float qd, f;
+            const float g = term(d, qd, f) ? f + 1.f : 0.f;
+            grad[d] = qd * (g - gbar);
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t od_launch_distill(od_ctx *c, int32_t B, int32_t K_max, const float *q_rows,
+                              const int32_t *draft_ids, const int32_t *tgt_ids, const int32_t *span_start,
+                              const int32_t *span_len, const int32_t *m, const void *logits, int32_t dtype,
+                              int64_t row_stride, int64_t seq_stride, const float *row_max,
+                              const float *row_sum, const float *p_sel, const float *temperature,
+                              float lambda, int32_t lambda_mode, float *loss, float *grad, cudaStream_t s)
+{
+    if (B == 0) return cudaSuccess;
+    DistillArgs a;
+    a.B = B; a.K_max = K_max; a.v_q = c->v_q; a.v_p = c->v_p;
+    a.q_rows = q_rows; a.draft_ids = draft_ids; a.tgt_ids = tgt_ids; a.span_start = span_start;
+    a.span_len = span_len; a.m = m; a.logits = logits; a.row_stride = row_stride; a.seq_stride = seq_stride;
+    a.row_max = row_max; a.row_sum = row_sum; a.p_sel = p_sel; a.temperature = temperature;
+    a.vocab_map = c->d_vocab_map; a.lambda = lambda; a.lambda_mode = lambda_mode; a.loss = loss; a.grad = grad;
+    dim3 grid((unsigned)K_max, (unsigned)B);
+    if (dtype == OD_BF16) od_distill_kernel<OD_BF16><<<grid, THREADS, 0, s>>>(a);
+    else od_distill_kernel<OD_F32><<<grid, THREADS, 0, s>>>(a);
+    return cudaGetLastError();
+}
