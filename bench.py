@@ -307,7 +307,10 @@ def run_distill(a):
     ms = e0.elapsed_time(e1) / a.steps
     active = sum(int(mps[i % P].span_len[torch.arange(K, device=dev)[None, :] < mps[i % P].m[:, None]].sum())
                  for i in range(a.steps)) / a.steps
-    bytes_per_call = active * 2 * w.v_q * 4 + (B * K - active) * w.v_q * 4
+    # active position: drafter row in, gradient row out, and (for the KL positions, nearly all) the target
+    # row, whose gathered ids touch practically every 32-byte sector; other positions: zeros out
+    esz_l = pool[0].logits.element_size()
+    bytes_per_call = active * (2 * w.v_q * 4 + w.v_p * esz_l) + (B * K - active) * w.v_q * 4
     peak, peak_src = measured_peak()
     print(json.dumps({
         "metric": "distilled_draft_positions_per_sec", "value": active / (ms * 1e-3), "unit": "positions/s",

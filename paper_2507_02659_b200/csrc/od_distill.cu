@@ -12,17 +12,19 @@
 // ln p_i(t) = (x_t - M_i)/T - ln S_i reuses the row statistics od_verify produced, so
 // the target row is only gathered at the mapped ids, never streamed again.
 //
-// One block of 1024 threads per (sequence, draft position); two sweeps over the draft
-// vocabulary (sums, then gradient; the second sweep finds its inputs in cache), reads
-// coalesced except the one gathered logit per mapped id. Bound by HBM: the drafter's
-// row in, the gradient row out.
+// One block of 512 threads per (sequence, draft position), two resident per SM so
+// that a whole batch is one wave; two sweeps over the draft vocabulary: sums, with
+// q(d) g(d) parked in the gradient row, then the gradient (which re-reads q and the
+// parked values from cache). Reads are coalesced except the one gathered logit per
+// mapped id, which touches practically every sector of the target row. Bound by HBM:
+// the drafter's row and the target row in, the gradient row out.
 #include <float.h>
 
 #include "od_common.cuh"
 
 namespace {
 
-constexpr int THREADS = 1024;
+constexpr int THREADS = 512;
 
 struct DistillArgs {
     int32_t B, K_max, v_q, v_p;
@@ -36,6 +38,15 @@ struct DistillArgs {
     int32_t lambda_mode;
     float *loss, *grad;
 };
+
+// log2 on the special-function unit (relative error about 2^-22; the terms it enters are
+// weighted by q, so the loss and the gradient see it far below their fp32 rounding)
+__device__ __forceinline__ float lg2_approx(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 __device__ __forceinline__ double block_sum(double v, double *s_red)
 {
@@ -60,11 +71,16 @@ od_distill_kernel(const DistillArgs a)
     int mb = a.m[b];
     mb = mb < 0 ? 0 : (mb > K ? K : mb);
     // the piece of the translated proposal that covers draft position j, if any
-    int piece = -1, plen = 0;
-    for (int i = 0; i < mb; ++i) {
-        const int s0 = a.span_start[(size_t)b * K + i], L = a.span_len[(size_t)b * K + i];
-        if (j >= s0 && j < s0 + L) { piece = i; plen = L; }
+    // (thread i looks at piece i, so the loads go out together)
+    __shared__ int s_piece, s_plen;
+    if (threadIdx.x == 0) { s_piece = -1; s_plen = 0; }
+    __syncthreads();
+    if ((int)threadIdx.x < mb) {
+        const int s0 = a.span_start[(size_t)b * K + threadIdx.x], L = a.span_len[(size_t)b * K + threadIdx.x];
+        if (j >= s0 && j < s0 + L) { s_piece = (int)threadIdx.x; s_plen = L; }
     }
+    __syncthreads();
+    const int piece = s_piece, plen = s_plen;
     const float *q = a.q_rows + ((size_t)b * K + j) * a.v_q;
     float *grad = a.grad ? a.grad + ((size_t)b * K + j) * a.v_q : nullptr;
     const float T = a.temperature[b];
@@ -86,34 +102,62 @@ od_distill_kernel(const DistillArgs a)
     // ---- a directly mapped token: KL(q' || p_i) over the mapped ids
     const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
     const char *row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)piece * a.row_stride) * esz;
+    // The gathers below touch practically every 32-byte sector of the target row in no
+    // particular order: have the copy engine bring the row into L2 as one sequential
+    // transfer first (a no-op when od_verify has just streamed it).
+    if (threadIdx.x == 0) {
+        const uint32_t bytes = (uint32_t)((size_t)a.v_p * esz / 16 * 16);
+        if (bytes) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
+    }
+    // in base 2: ln q - ln p(t) = ln 2 * (lg2 q - ((x_t - M) * log2(e)/T - lg2 S))
     const float M = a.row_max[b * (K + 1) + piece];
-    const float ln_S = logf(a.row_sum[b * (K + 1) + piece]);
-    const float inv_T = 1.f / T;
-    // f(d) = ln q(d) - ln p(map[d]) for a mapped d with q(d) > 0, else "no term"
-    auto term = [&](int d, float &qd, float &f) -> bool {
-        const int32_t t = __ldg(a.vocab_map + d);
-        qd = __ldg(q + d);
-        if (t < 0 || !(qd > 0.f)) return false;
-        f = logf(qd) - ((od_load_logit<DTYPE>(row, t) - M) * inv_T - ln_S);
-        return true;
-    };
-    float loss_t = 0.f, qg_t = 0.f;                          // sum q f, sum q (f + 1) over this thread's ids
-#pragma unroll 4
-    for (int d = threadIdx.x; d < a.v_q; d += THREADS) {
-        float qd, f;
-        if (term(d, qd, f)) { loss_t += qd * f; qg_t += qd * (f + 1.f); }
+    const float lg2_S = lg2_approx(a.row_sum[b * (K + 1) + piece]);
+    const float scale = 1.4426950408889634f / T;
+    constexpr float LN2 = 0.6931471805599453f;
+    // Sweep 1: g(d) = [d mapped, q(d) > 0] (ln q(d) - ln p(map[d]) + 1), the loss and
+    // sum_d q(d) g(d). The loads of EB ids are issued together (map and q, then the
+    // gathered logits). q(d) g(d) is parked in the gradient row itself (it stays in L2),
+    // so that sweep 2 neither gathers nor takes a logarithm again.
+    constexpr int EB = 16;
+    const bool park = grad != nullptr;
+    float loss_t = 0.f, qg_t = 0.f;
+    for (int base = threadIdx.x; base < a.v_q; base += THREADS * EB) {
+        float qd[EB], x[EB];
+        {
+            int32_t t[EB];
+#pragma unroll
+            for (int e = 0; e < EB; ++e) {
+                const int d = base + e * THREADS;
+                t[e] = d < a.v_q ? __ldg(a.vocab_map + d) : -1;
+                qd[e] = d < a.v_q ? __ldg(q + d) : 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < EB; ++e)                     // an id without a map: q = 0 drops its term below
+                if (t[e] < 0) qd[e] = -qd[e];
+#pragma unroll
+            for (int e = 0; e < EB; ++e) x[e] = od_load_logit<DTYPE>(row, t[e] >= 0 ? t[e] : 0);
+        }
+#pragma unroll
+        for (int e = 0; e < EB; ++e) {
+            const int d = base + e * THREADS;
+            const bool ok = qd[e] >= FLT_MIN;                // mapped and with (normal) mass
+            qd[e] = fabsf(qd[e]);
+            const float f = ok ? LN2 * (lg2_approx(qd[e]) - fmaf(x[e] - M, scale, -lg2_S)) : 0.f;
+            const float g = ok ? f + 1.f : 0.f;
+            loss_t += qd[e] * f;
+            qg_t += qd[e] * g;
+            if (park && d < a.v_q) grad[d] = qd[e] * g;
+        }
     }
     const double loss = block_sum((double)loss_t, s_red);
     const double qg = block_sum((double)qg_t, s_red);
     if (threadIdx.x == 0) a.loss[(size_t)b * K + j] = (float)loss;
     if (grad) {
+        // Sweep 2: grad(d) = q(d) g(d) - q(d) * sum_e q(e) g(e); every thread revisits the
+        // ids it wrote itself, so no barrier is needed for the parked values
         const float gbar = (float)qg;
 #pragma unroll 4
-        for (int d = threadIdx.x; d < a.v_q; d += THREADS) {
-            float qd, f;
-            const float g = term(d, qd, f) ? f + 1.f : 0.f;
-            grad[d] = qd * (g - gbar);
-        }
+        for (int d = threadIdx.x; d < a.v_q; d += THREADS) grad[d] = fmaf(-__ldg(q + d), gbar, grad[d]);
     }
 }
 
