@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the cross-vocabulary verification step (one JSON line).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..6] [--impl reference]
 
 A step is one pass of the whole hot path (od_map_proposals -> od_verify ->
 od_sample_residual) over one batch of synthetic input. The default workload is

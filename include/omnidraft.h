@@ -382,6 +382,89 @@ int32_t od_step_host(od_ctx *ctx, int32_t B, int32_t K_max,
                      int32_t *tgt_ids, int32_t *m, uint32_t *verify_flags,
                      uint32_t *sample_flags, void *stream);
 
+/* ---- the step with the target vocabulary split over GPUs ------------------ */
+
+/* Steps 2 and 3 when the target model's output layer is split by columns over
+ * n_shards GPUs (tensor parallelism): every GPU holds, for all rows, the logits of
+ * the target ids [shard_lo, shard_lo + shard_len) only. The paper runs the target on
+ * one GPU and has no counterpart of the split; the result is Algorithm 1's and
+ * Eq. (2)'s, unchanged, because a row's softmax statistics and the residual's
+ * cumulative sums are sums over disjoint id ranges. A step is
+ *   od_verify_shard_stats   -> exchange (all-gather, the caller's) ->
+ *   od_verify_shard_finish  -> od_sample_shard_mass -> exchange ->
+ *   od_sample_shard_pick    -> exchange of the B picked tokens,
+ * with the same od_map_proposals outputs, temperatures and seeds on every GPU, so
+ * that all GPUs take identical decisions. Every context is created with the FULL
+ * target vocabulary, map and cache. Shards must tile the vocabulary in id order;
+ * shard_lo must be a multiple of 256 and shard_lo + shard_len either a multiple of
+ * 256 or the vocabulary size (INVALID_ARG otherwise). `logits` points at the
+ * shard's own buffer: element (b, r, shard_lo + c) at b*seq_stride + r*row_stride + c,
+ * row_stride >= shard_len, alignment as for od_verify. All four calls are
+ * asynchronous on `stream` and allocate nothing. */
+
+/* Per-row statistics of this shard's columns (Algorithm 1, target-probability line,
+ * restricted to the shard): stats[(b*(K_max+1) + r)*4 + 0..3] = (c, s, M, x) for rows
+ * r <= m_b, where M is the exact maximum of the shard's logits of the row, c a
+ * reference exponent in the scaled domain (c >= M*log2(e)/T_b up to rounding),
+ * s = sum over the shard of exp2(x*log2(e)/T_b - c), and x = the logit of t_r if this
+ * shard owns it (r < m_b), else -inf. Other rows are left untouched.
+ *   in  (device) logits (the shard's), tgt_ids, m from od_map_proposals, temperature
+ *   out (device) stats float[B*(K_max+1)*4], 16-byte aligned */
+int32_t od_verify_shard_stats(od_ctx *ctx, int32_t B, int32_t K_max, int32_t shard_lo,
+                              int32_t shard_len, const void *logits, int32_t logit_dtype,
+                              int64_t row_stride, int64_t seq_stride,
+                              const int32_t *tgt_ids, const int32_t *m,
+                              const float *temperature, float *stats, void *stream);
+
+/* Merges the records of all shards (stats_all = the n_shards stats arrays one after
+ * the other, in shard order) and produces exactly the outputs of od_verify
+ * (1 <= n_shards <= 1024). Deterministic: every GPU gets the same bits. */
+int32_t od_verify_shard_finish(od_ctx *ctx, int32_t B, int32_t K_max, int32_t n_shards,
+                               const float *stats_all, const int32_t *tgt_ids,
+                               const float *q_prime, const int32_t *span_len,
+                               const int32_t *m, const float *temperature,
+                               const uint64_t *seed, uint64_t step, float *row_max,
+                               float *row_sum, float *p_sel, float *ratio,
+                               int32_t *n_accepted, int32_t *n_draft_accepted,
+                               uint32_t *verify_flags, void *stream);
+
+/* This shard's share of the mass the extra token is drawn from (arguments as for
+ * od_sample_residual, row_max / row_sum / n_accepted from od_verify_shard_finish):
+ * mass[2b] = sum over the shard's ids of r(t) (unnormalised: times the row sum),
+ * mass[2b+1] = the shard's share of p_j in the same units if mass[2b] is zero for a
+ * residual draw (needed when no shard has residual mass), else 0.
+ *   out (device) mass double[B*2] */
+int32_t od_sample_shard_mass(od_ctx *ctx, int32_t B, int32_t K_max, int32_t shard_lo,
+                             int32_t shard_len, const void *logits, int32_t logit_dtype,
+                             int64_t row_stride, int64_t seq_stride, const float *row_max,
+                             const float *row_sum, const float *q_rows,
+                             const int32_t *draft_ids, const int32_t *tgt_ids,
+                             const float *q_prime, const int32_t *span_start,
+                             const int32_t *span_len, const int32_t *m,
+                             const uint8_t *tail_kind, const int32_t *n_accepted,
+                             const float *temperature, double *mass, void *stream);
+
+/* The draw, after the shares of all shards were exchanged (mass_all = the n_shards
+ * mass arrays in shard order; must follow od_sample_shard_mass of the same step on
+ * this context, which leaves the shard's tile sums in the context's scratch). The
+ * inverse-CDF walk of od_sample_residual runs over the shards in id order and, inside
+ * the shard it stops in, over that shard's ids. Exactly one shard writes the token:
+ * the others write out_token = -1, resid_mass = 0, sample_flags = 0, so that the
+ * element-wise maximum (tokens, masses) and OR (flags) over the shards is the result
+ * of od_sample_residual. */
+int32_t od_sample_shard_pick(od_ctx *ctx, int32_t B, int32_t K_max, int32_t n_shards,
+                             int32_t shard_index, int32_t shard_lo, int32_t shard_len,
+                             const double *mass_all, const void *logits,
+                             int32_t logit_dtype, int64_t row_stride, int64_t seq_stride,
+                             const float *row_max, const float *row_sum,
+                             const float *q_rows, const int32_t *draft_ids,
+                             const int32_t *tgt_ids, const float *q_prime,
+                             const int32_t *span_start, const int32_t *span_len,
+                             const int32_t *m, const uint8_t *tail_kind,
+                             const int32_t *n_accepted, const float *temperature,
+                             const uint64_t *seed, uint64_t step, int32_t *out_token,
+                             float *resid_mass, uint32_t *sample_flags, void *stream);
+
 /* ---- misc ---------------------------------------------------------------- */
 
 /* Launch shape of the last od_verify / od_sample_residual call on this context

@@ -19,6 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libomnidraft.so")
 
 OD_F32, OD_BF16 = 0, 1
+OD_ERR_INVALID_ARG, OD_ERR_ALIGNMENT = -1, -2
 OD_TAIL_COMPLETE, OD_TAIL_UNMAPPED_STOP = 0, 1
 OD_CNT_CACHE_HITS, OD_CNT_UNMAPPED_STOPS, OD_CNT_INVALID_IDS, OD_CNT_MAPPED_TOKENS = 0, 1, 2, 3
 OD_CNT_COUNT = 4
@@ -31,7 +32,9 @@ OD_NOALLOC_MAX_ROWS = 1024
 EXPORTS = ["od_create", "od_destroy", "od_set_vocab_map", "od_cache_build", "od_set_option",
            "od_map_proposals", "od_verify", "od_sample_residual", "od_host_step_reserve",
            "od_step_host", "od_verify_noalloc", "od_exit_rule", "od_cache_configure", "od_cache_set_clock",
-           "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_distill_loss", "od_last_launch_info", "od_status_string", "od_version"]
+           "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_distill_loss",
+           "od_verify_shard_stats", "od_verify_shard_finish", "od_sample_shard_mass", "od_sample_shard_pick",
+           "od_last_launch_info", "od_status_string", "od_version"]
 
 
 class OdError(RuntimeError):
@@ -67,6 +70,11 @@ def lib():
         L.od_exit_rule.argtypes = [vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp]
         L.od_distill_loss.argtypes = ([vp, i32, i32] + [vp] * 7 + [i32, i64, i64] + [vp] * 4
                                       + [C.c_float, i32, vp, vp, vp])
+        L.od_verify_shard_stats.argtypes = [vp, i32, i32, i32, i32, vp, i32, i64, i64] + [vp] * 4 + [vp]
+        L.od_verify_shard_finish.argtypes = [vp, i32, i32, i32] + [vp] * 7 + [u64] + [vp] * 7 + [vp]
+        L.od_sample_shard_mass.argtypes = [vp, i32, i32, i32, i32, vp, i32, i64, i64] + [vp] * 12 + [vp] + [vp]
+        L.od_sample_shard_pick.argtypes = ([vp, i32, i32, i32, i32, i32, i32, vp, vp, i32, i64, i64] + [vp] * 13
+                                           + [u64] + [vp] * 3 + [vp])
         L.od_cache_configure.argtypes = [vp, i64, i32, i32]
         L.od_cache_set_clock.argtypes = [vp, C.c_uint32]
         L.od_cache_insert.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -361,6 +369,96 @@ def od_sample_residual(ctx: Context, logits, vo: VerifyOut, q_rows, draft_ids, m
         _dp(seed, torch.int64, d), C.c_uint64(step & (2**64 - 1)),
         _dp(out.out_token, i32, d), _dp(out.resid_mass, f32, d), _dp(out.flags, i32, d),
         _stream(d)), "od_sample_residual")
+    return out
+
+
+# ---- the step with the target vocabulary split over GPUs (one call per phase) ----
+
+def _shard_strides(logits: torch.Tensor, B: int, K: int, shard_len: int):
+    if logits.dim() != 3 or logits.shape[0] != B or logits.shape[1] != K + 1 or logits.shape[2] != shard_len:
+        raise ValueError(f"shard logits must be [B, K+1, shard_len], got {tuple(logits.shape)}")
+    if logits.stride(2) != 1:
+        raise ValueError("logit rows must be dense")
+    return int(logits.stride(1)), int(logits.stride(0))
+
+
+def od_verify_shard_stats(ctx: Context, shard_lo: int, logits, mp: MapOut, temperature,
+                          out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Per-row records (c, s, M, x[t]) of this shard's columns: float32 [B, K+1, 4]."""
+    B, K = mp.tgt_ids.shape
+    d, i32, f32 = ctx.device, torch.int32, torch.float32
+    shard_len = int(logits.shape[2])
+    rs, ss = _shard_strides(logits, B, K, shard_len)
+    if out is None:
+        out = torch.zeros(B, K + 1, 4, dtype=f32, device=d)
+    _check(lib().od_verify_shard_stats(
+        ctx.handle, B, K, shard_lo, shard_len, C.c_void_p(logits.data_ptr()), logit_dtype_code(logits),
+        rs, ss, _dp(mp.tgt_ids, i32, d), _dp(mp.m, i32, d), _dp(temperature, f32, d), _dp(out, f32, d),
+        _stream(d)), "od_verify_shard_stats")
+    return out
+
+
+def od_verify_shard_finish(ctx: Context, stats_all: torch.Tensor, mp: MapOut, temperature, seed, step: int,
+                           out: Optional[VerifyOut] = None) -> VerifyOut:
+    """stats_all: float32 [n_shards, B, K+1, 4], shard order."""
+    B, K = mp.tgt_ids.shape
+    if stats_all.dim() != 4 or tuple(stats_all.shape[1:]) != (B, K + 1, 4):
+        raise ValueError("stats_all must be [n_shards, B, K+1, 4]")
+    out = out or alloc_verify_out(ctx, B, K)
+    d, i32, f32 = ctx.device, torch.int32, torch.float32
+    _check(lib().od_verify_shard_finish(
+        ctx.handle, B, K, int(stats_all.shape[0]), _dp(stats_all, f32, d),
+        _dp(mp.tgt_ids, i32, d), _dp(mp.q_prime, f32, d), _dp(mp.span_len, i32, d), _dp(mp.m, i32, d),
+        _dp(temperature, f32, d), _dp(seed, torch.int64, d), C.c_uint64(step & (2**64 - 1)),
+        _dp(out.row_max, f32, d), _dp(out.row_sum, f32, d), _dp(out.p_sel, f32, d),
+        _dp(out.ratio, f32, d), _dp(out.n_accepted, i32, d), _dp(out.n_draft_accepted, i32, d),
+        _dp(out.flags, i32, d), _stream(d)), "od_verify_shard_finish")
+    return out
+
+
+def od_sample_shard_mass(ctx: Context, shard_lo: int, logits, vo: VerifyOut, q_rows, draft_ids, mp: MapOut,
+                         temperature, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """This shard's shares of the sampling mass: float64 [B, 2]."""
+    B, K = mp.tgt_ids.shape
+    d, i32, f32 = ctx.device, torch.int32, torch.float32
+    shard_len = int(logits.shape[2])
+    rs, ss = _shard_strides(logits, B, K, shard_len)
+    if tuple(q_rows.shape) != (B, K, ctx.draft_vocab):
+        raise ValueError("q_rows must be [B, K, V_q]")
+    if out is None:
+        out = torch.zeros(B, 2, dtype=torch.float64, device=d)
+    _check(lib().od_sample_shard_mass(
+        ctx.handle, B, K, shard_lo, shard_len, C.c_void_p(logits.data_ptr()), logit_dtype_code(logits),
+        rs, ss, _dp(vo.row_max, f32, d), _dp(vo.row_sum, f32, d), _dp(q_rows, f32, d),
+        _dp(draft_ids, i32, d), _dp(mp.tgt_ids, i32, d), _dp(mp.q_prime, f32, d),
+        _dp(mp.span_start, i32, d), _dp(mp.span_len, i32, d), _dp(mp.m, i32, d),
+        _dp(mp.tail_kind, torch.uint8, d), _dp(vo.n_accepted, i32, d), _dp(temperature, f32, d),
+        _dp(out, torch.float64, d), _stream(d)), "od_sample_shard_mass")
+    return out
+
+
+def od_sample_shard_pick(ctx: Context, shard_index: int, shard_lo: int, mass_all: torch.Tensor, logits,
+                         vo: VerifyOut, q_rows, draft_ids, mp: MapOut, temperature, seed, step: int,
+                         out: Optional[SampleOut] = None) -> SampleOut:
+    """mass_all: float64 [n_shards, B, 2], shard order. Only the shard that holds the
+    token writes it; the others write (-1, 0, 0)."""
+    B, K = mp.tgt_ids.shape
+    if mass_all.dim() != 3 or tuple(mass_all.shape[1:]) != (B, 2):
+        raise ValueError("mass_all must be [n_shards, B, 2]")
+    out = out or alloc_sample_out(ctx, B)
+    d, i32, f32 = ctx.device, torch.int32, torch.float32
+    shard_len = int(logits.shape[2])
+    rs, ss = _shard_strides(logits, B, K, shard_len)
+    _check(lib().od_sample_shard_pick(
+        ctx.handle, B, K, int(mass_all.shape[0]), shard_index, shard_lo, shard_len,
+        _dp(mass_all, torch.float64, d), C.c_void_p(logits.data_ptr()), logit_dtype_code(logits), rs, ss,
+        _dp(vo.row_max, f32, d), _dp(vo.row_sum, f32, d), _dp(q_rows, f32, d),
+        _dp(draft_ids, i32, d), _dp(mp.tgt_ids, i32, d), _dp(mp.q_prime, f32, d),
+        _dp(mp.span_start, i32, d), _dp(mp.span_len, i32, d), _dp(mp.m, i32, d),
+        _dp(mp.tail_kind, torch.uint8, d), _dp(vo.n_accepted, i32, d), _dp(temperature, f32, d),
+        _dp(seed, torch.int64, d), C.c_uint64(step & (2**64 - 1)),
+        _dp(out.out_token, i32, d), _dp(out.resid_mass, f32, d), _dp(out.flags, i32, d),
+        _stream(d)), "od_sample_shard_pick")
     return out
 
 

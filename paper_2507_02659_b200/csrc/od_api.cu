@@ -67,15 +67,32 @@ int32_t check_step_common(const od_ctx *c, int32_t B, int32_t K_max)
     return OD_OK;
 }
 
-int32_t check_logits(const od_ctx *c, const void *logits, int32_t dtype, int64_t row_stride,
-                     int64_t seq_stride, int32_t K_max)
+// row_len: elements of a row (the whole vocabulary, or a shard's columns)
+int32_t check_logits_len(int64_t row_len, const void *logits, int32_t dtype, int64_t row_stride,
+                         int64_t seq_stride, int32_t K_max)
 {
     if (!logits) return OD_ERR_INVALID_ARG;
     if (dtype != OD_F32 && dtype != OD_BF16) return OD_ERR_UNSUPPORTED;
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
-    if (row_stride < c->v_p || seq_stride < row_stride * (K_max + 1)) return OD_ERR_INVALID_ARG;
+    if (row_stride < row_len || seq_stride < row_stride * (K_max + 1)) return OD_ERR_INVALID_ARG;
     if (!aligned16(logits) || (row_stride * esz) % 16 != 0 || (seq_stride * esz) % 16 != 0)
         return OD_ERR_ALIGNMENT;
+    return OD_OK;
+}
+
+int32_t check_logits(const od_ctx *c, const void *logits, int32_t dtype, int64_t row_stride,
+                     int64_t seq_stride, int32_t K_max)
+{
+    return check_logits_len(c->v_p, logits, dtype, row_stride, seq_stride, K_max);
+}
+
+// a vocabulary shard: whole 256-id tiles, inside the vocabulary
+int32_t check_shard(const od_ctx *c, int32_t shard_lo, int32_t shard_len)
+{
+    if (shard_lo < 0 || shard_len < 1 || (int64_t)shard_lo + shard_len > c->v_p) return OD_ERR_INVALID_ARG;
+    if (shard_lo % OD_SAMPLE_TILE != 0) return OD_ERR_INVALID_ARG;
+    const int32_t hi = shard_lo + shard_len;
+    if (hi % OD_SAMPLE_TILE != 0 && hi != c->v_p) return OD_ERR_INVALID_ARG;
     return OD_OK;
 }
 
@@ -320,6 +337,106 @@ int32_t od_sample_residual(od_ctx *c, int32_t B, int32_t K_max, const void *logi
                              row_sum, q_rows, draft_ids, tgt_ids, q_prime, span_start, span_len, m,
                              tail_kind, n_accepted, temperature, seed, step, out_token, resid_mass,
                              sample_flags, (cudaStream_t)stream));
+    return OD_OK;
+}
+
+int32_t od_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo, int32_t shard_len,
+                              const void *logits, int32_t logit_dtype, int64_t row_stride,
+                              int64_t seq_stride, const int32_t *tgt_ids, const int32_t *m,
+                              const float *temperature, float *stats, void *stream)
+{
+    int32_t st = check_step_common(c, B, K_max);
+    if (st != OD_OK) return st;
+    st = check_shard(c, shard_lo, shard_len);
+    if (st != OD_OK) return st;
+    st = check_logits_len(shard_len, logits, logit_dtype, row_stride, seq_stride, K_max);
+    if (st != OD_OK) return st;
+    if (!tgt_ids || !m || !temperature || !stats) return OD_ERR_INVALID_ARG;
+    if (!aligned16(stats)) return OD_ERR_ALIGNMENT;
+    DeviceGuard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    OD_CUDA(od_launch_verify_shard_stats(c, B, K_max, shard_lo, shard_len, logits, logit_dtype, row_stride,
+                                         seq_stride, tgt_ids, m, temperature, stats, (cudaStream_t)stream));
+    return OD_OK;
+}
+
+int32_t od_verify_shard_finish(od_ctx *c, int32_t B, int32_t K_max, int32_t n_shards,
+                               const float *stats_all, const int32_t *tgt_ids, const float *q_prime,
+                               const int32_t *span_len, const int32_t *m, const float *temperature,
+                               const uint64_t *seed, uint64_t step, float *row_max, float *row_sum,
+                               float *p_sel, float *ratio, int32_t *n_accepted,
+                               int32_t *n_draft_accepted, uint32_t *verify_flags, void *stream)
+{
+    int32_t st = check_step_common(c, B, K_max);
+    if (st != OD_OK) return st;
+    if (n_shards < 1 || n_shards > 1024) return OD_ERR_INVALID_ARG;
+    if (!stats_all || !tgt_ids || !q_prime || !span_len || !m || !temperature || !seed || !row_max ||
+        !row_sum || !p_sel || !ratio || !n_accepted || !n_draft_accepted || !verify_flags)
+        return OD_ERR_INVALID_ARG;
+    if (!aligned16(stats_all)) return OD_ERR_ALIGNMENT;
+    DeviceGuard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    OD_CUDA(od_launch_verify_shard_finish(c, B, K_max, n_shards, stats_all, tgt_ids, q_prime, span_len, m,
+                                          temperature, seed, step, row_max, row_sum, p_sel, ratio,
+                                          n_accepted, n_draft_accepted, verify_flags, (cudaStream_t)stream));
+    return OD_OK;
+}
+
+int32_t od_sample_shard_mass(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo, int32_t shard_len,
+                             const void *logits, int32_t logit_dtype, int64_t row_stride,
+                             int64_t seq_stride, const float *row_max, const float *row_sum,
+                             const float *q_rows, const int32_t *draft_ids, const int32_t *tgt_ids,
+                             const float *q_prime, const int32_t *span_start, const int32_t *span_len,
+                             const int32_t *m, const uint8_t *tail_kind, const int32_t *n_accepted,
+                             const float *temperature, double *mass, void *stream)
+{
+    int32_t st = check_step_common(c, B, K_max);
+    if (st != OD_OK) return st;
+    st = check_shard(c, shard_lo, shard_len);
+    if (st != OD_OK) return st;
+    st = check_logits_len(shard_len, logits, logit_dtype, row_stride, seq_stride, K_max);
+    if (st != OD_OK) return st;
+    if (!row_max || !row_sum || !q_rows || !draft_ids || !tgt_ids || !q_prime || !span_start ||
+        !span_len || !m || !tail_kind || !n_accepted || !temperature || !mass)
+        return OD_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    OD_CUDA(od_launch_sample_shard_mass(c, B, K_max, shard_lo, shard_len, logits, logit_dtype, row_stride,
+                                        seq_stride, row_max, row_sum, q_rows, draft_ids, tgt_ids, q_prime,
+                                        span_start, span_len, m, tail_kind, n_accepted, temperature, mass,
+                                        (cudaStream_t)stream));
+    return OD_OK;
+}
+
+int32_t od_sample_shard_pick(od_ctx *c, int32_t B, int32_t K_max, int32_t n_shards, int32_t shard_index,
+                             int32_t shard_lo, int32_t shard_len, const double *mass_all,
+                             const void *logits, int32_t logit_dtype, int64_t row_stride,
+                             int64_t seq_stride, const float *row_max, const float *row_sum,
+                             const float *q_rows, const int32_t *draft_ids, const int32_t *tgt_ids,
+                             const float *q_prime, const int32_t *span_start, const int32_t *span_len,
+                             const int32_t *m, const uint8_t *tail_kind, const int32_t *n_accepted,
+                             const float *temperature, const uint64_t *seed, uint64_t step,
+                             int32_t *out_token, float *resid_mass, uint32_t *sample_flags, void *stream)
+{
+    int32_t st = check_step_common(c, B, K_max);
+    if (st != OD_OK) return st;
+    if (n_shards < 1 || n_shards > 1024 || shard_index < 0 || shard_index >= n_shards)
+        return OD_ERR_INVALID_ARG;
+    st = check_shard(c, shard_lo, shard_len);
+    if (st != OD_OK) return st;
+    st = check_logits_len(shard_len, logits, logit_dtype, row_stride, seq_stride, K_max);
+    if (st != OD_OK) return st;
+    if (!mass_all || !row_max || !row_sum || !q_rows || !draft_ids || !tgt_ids || !q_prime ||
+        !span_start || !span_len || !m || !tail_kind || !n_accepted || !temperature || !seed ||
+        !out_token || !resid_mass || !sample_flags)
+        return OD_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    OD_CUDA(od_launch_sample_shard_pick(c, B, K_max, n_shards, shard_index, shard_lo, shard_len, mass_all,
+                                        logits, logit_dtype, row_stride, seq_stride, row_max, row_sum,
+                                        q_rows, draft_ids, tgt_ids, q_prime, span_start, span_len, m,
+                                        tail_kind, n_accepted, temperature, seed, step, out_token,
+                                        resid_mass, sample_flags, (cudaStream_t)stream));
     return OD_OK;
 }
 

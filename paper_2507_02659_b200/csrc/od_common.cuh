@@ -106,6 +106,38 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
                              cudaStream_t s);
 
+// vocabulary shards (columns [shard_lo, shard_lo + shard_len) of the rows on this GPU)
+cudaError_t od_launch_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo,
+                                         int32_t shard_len, const void *logits, int32_t dtype,
+                                         int64_t row_stride, int64_t seq_stride, const int32_t *tgt_ids,
+                                         const int32_t *m, const float *temperature, float *stats,
+                                         cudaStream_t s);
+cudaError_t od_launch_verify_shard_finish(od_ctx *c, int32_t B, int32_t K_max, int32_t n_shards,
+                                          const float *stats_all, const int32_t *tgt_ids,
+                                          const float *q_prime, const int32_t *span_len, const int32_t *m,
+                                          const float *temperature, const uint64_t *seed, uint64_t step,
+                                          float *row_max, float *row_sum, float *p_sel, float *ratio,
+                                          int32_t *n_accepted, int32_t *n_draft_accepted, uint32_t *flags,
+                                          cudaStream_t s);
+cudaError_t od_launch_sample_shard_mass(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo,
+                                        int32_t shard_len, const void *logits, int32_t dtype,
+                                        int64_t row_stride, int64_t seq_stride, const float *row_max,
+                                        const float *row_sum, const float *q_rows, const int32_t *draft_ids,
+                                        const int32_t *tgt_ids, const float *q_prime,
+                                        const int32_t *span_start, const int32_t *span_len, const int32_t *m,
+                                        const uint8_t *tail_kind, const int32_t *n_accepted,
+                                        const float *temperature, double *mass, cudaStream_t s);
+cudaError_t od_launch_sample_shard_pick(od_ctx *c, int32_t B, int32_t K_max, int32_t n_shards,
+                                        int32_t shard_index, int32_t shard_lo, int32_t shard_len,
+                                        const double *mass_all, const void *logits, int32_t dtype,
+                                        int64_t row_stride, int64_t seq_stride, const float *row_max,
+                                        const float *row_sum, const float *q_rows, const int32_t *draft_ids,
+                                        const int32_t *tgt_ids, const float *q_prime,
+                                        const int32_t *span_start, const int32_t *span_len, const int32_t *m,
+                                        const uint8_t *tail_kind, const int32_t *n_accepted,
+                                        const float *temperature, const uint64_t *seed, uint64_t step,
+                                        int32_t *out_token, float *resid_mass, uint32_t *flags, cudaStream_t s);
+
 cudaError_t od_launch_distill(od_ctx *c, int32_t B, int32_t K_max, const float *q_rows,
                               const int32_t *draft_ids, const int32_t *tgt_ids, const int32_t *span_start,
                               const int32_t *span_len, const int32_t *m, const void *logits, int32_t dtype,

@@ -27,6 +27,16 @@
 // Sums and scans across lanes and tiles are fp64 in a fixed order: the result is
 // reproducible, and the only difference to exact arithmetic is the fp32 rounding
 // of the individual terms.
+//
+// Vocabulary shards (the rows split by columns over several GPUs) use the same
+// kernel in two further modes. A shard owns a window of whole tiles:
+//   mode 1  pass 1 over the window, then the last block adds the window's tile
+//           values: the shard's share of the residual mass (and, when that is
+//           zero, of the mass of p_j, for the fallback);
+//   mode 2  after the shares of all shards were exchanged: every shard forms the
+//           same total and target = u * total, finds the shard in which the running
+//           sum over shards crosses the target, and that shard alone scans its
+//           window (offset by the shares before it) as in pass 2.
 #include <float.h>
 
 #include "od_common.cuh"
@@ -58,6 +68,12 @@ struct SampleArgs {
     int32_t list_width;
     double *tile_val;                   // [B][ntiles] sum over the tile of r'
     unsigned int *ticket;
+    // vocabulary shards: this shard's tiles are [tile_lo, tile_hi); `logits` points at
+    // its first column (target id col0), v_p is the id one past its last column
+    int32_t tile_lo, tile_hi, col0;
+    int32_t n_shards, shard_index;
+    const double *mass_all;             // [n_shards][B][2] (residual share, share of p_j or 0)
+    double *mass_out;                   // [B][2] this shard's shares
 };
 
 // what one sequence's warps need to evaluate r(t)
@@ -211,7 +227,7 @@ __device__ __forceinline__ float warp_sum_f32(float v)
 // list bounds, then list entries, then the gathered probabilities and logits).
 template <int DTYPE, int TB>
 __device__ __forceinline__ void warp_batch(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
-                                           int n, int lane, double *tile_val)
+                                           int n, int lane, double *tile_val, int32_t dummy)
 {
     uint4 raw[TB][DTYPE == OD_BF16 ? 1 : 2];
     const int whole_n = (a.v_p / OD_SAMPLE_TILE - t_lo) < n ? (a.v_p / OD_SAMPLE_TILE - t_lo) : n;   // tiles with all 256 ids
@@ -243,7 +259,7 @@ __device__ __forceinline__ void warp_batch(const SeqState &q, const SampleArgs &
     for (int i = 0; i < TB; ++i) {
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-            const int32_t t = et[i][k] >= 0 ? et[i][k] : 0;   // always a valid address; the term is dropped below
+            const int32_t t = et[i][k] >= 0 ? et[i][k] : dummy;   // always a valid address; the term is dropped below
             ex[i][k] = od_load_logit<DTYPE>(q.row, t);
             eq[i][k] = __ldg(q.q_row + ed[i][k]);
         }
@@ -286,7 +302,7 @@ __device__ __forceinline__ void warp_batch(const SeqState &q, const SampleArgs &
                 for (int k = 2; k < rounds; ++k) {              // a wide list
                     const size_t idx = (size_t)(t_lo + i) * a.list_width + k * 32 + lane;
                     const int32_t t = __ldg(a.mapped_t + idx), d = __ldg(a.mapped_d + idx);
-                    sum -= corr_term<DTYPE>(q, t, d, od_load_logit<DTYPE>(q.row, t >= 0 ? t : 0), __ldg(q.q_row + d));
+                    sum -= corr_term<DTYPE>(q, t, d, od_load_logit<DTYPE>(q.row, t >= 0 ? t : dummy), __ldg(q.q_row + d));
                 }
                 // the n-gram's own token carries the n-gram's probability
                 if (lane == 0 && q.ngram_token >= 0 && q.ngram_token < a.v_p &&
@@ -303,14 +319,35 @@ __device__ __forceinline__ void warp_batch(const SeqState &q, const SampleArgs &
 
 template <int DTYPE>
 __device__ __forceinline__ void warp_tiles(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
-                                           int t_hi, int lane, double *tile_val)
+                                           int t_hi, int lane, double *tile_val, int32_t dummy)
 {
     constexpr int TB = 4;
     for (int t = t_lo; t < t_hi; t += TB)
-        warp_batch<DTYPE, TB>(q, a, residual, t, t_hi - t < TB ? t_hi - t : TB, lane, tile_val);
+        warp_batch<DTYPE, TB>(q, a, residual, t, t_hi - t < TB ? t_hi - t : TB, lane, tile_val, dummy);
 }
 
-template <int DTYPE>
+// Sum of s_val[my_lo, my_hi) over the block's threads in the order of the scan of
+// pass 2 (a thread's run, lanes in order, warps in order); every thread gets it.
+__device__ __forceinline__ double block_total(const double *s_val, int my_lo, int my_hi, double *s_warp)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double inc = 0.0;
+    for (int t = my_lo; t < my_hi; ++t) inc += s_val[t];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const double v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+        if (lane >= off) inc += v;
+    }
+    __syncthreads();                                // s_warp may still be read from an earlier call
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    double tot = 0.0;
+    for (int w = 0; w < WARPS; ++w) tot += s_warp[w];
+    return tot;
+}
+
+// MODE 0: the whole step on full rows; 1: a shard's mass shares; 2: a shard's pick.
+template <int DTYPE, int MODE>
 __global__ void __launch_bounds__(OD_SAMPLE_THREADS, 4)
 od_sample_kernel(const SampleArgs a)
 {
@@ -336,13 +373,23 @@ od_sample_kernel(const SampleArgs a)
     const float T = a.temperature[b];
     if (!(T > 0.f)) {                              // every block of the sequence leaves here
         if (blockIdx.x == 0 && threadIdx.x == 0) {
-            a.out_token[b] = -1; a.resid_mass[b] = 0.f; a.flags[b] = OD_SF_BAD_TEMPERATURE;
+            if (MODE == 1) {
+                a.mass_out[2 * b] = 0.0; a.mass_out[2 * b + 1] = 0.0;
+            } else {
+                a.out_token[b] = -1; a.resid_mass[b] = 0.f; a.flags[b] = OD_SF_BAD_TEMPERATURE;
+            }
         }
         return;
     }
     const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
+    // a shard's tiles and ids keep their numbers of the full row: the row pointer is
+    // moved back by the shard's first column, and only ids of the window are read
+    const int tile_lo = MODE == 0 ? 0 : a.tile_lo;
+    const int tile_hi = MODE == 0 ? a.ntiles : a.tile_hi;
+    const int32_t dummy = MODE == 0 ? 0 : tile_lo * OD_SAMPLE_TILE;   // an id that is safe to load
     SeqState q;
     q.row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)j * a.row_stride) * esz;
+    if (MODE != 0) q.row -= (size_t)a.col0 * esz;
     q.scale = 1.4426950408889634f / T;
     {
         // reference exponent c = fl(M*scale); the rounding of c goes into S exactly:
@@ -361,7 +408,7 @@ od_sample_kernel(const SampleArgs a)
         q.q_row = a.q_rows + ((size_t)b * K + s0) * a.v_q;
         // the gathers of pass 1 come two round trips from now: have the copy engine pull
         // this block's share of the drafter's row into L2 meanwhile
-        if (threadIdx.x == 0) {
+        if (MODE != 2 && threadIdx.x == 0) {
             const size_t row_bytes = (size_t)a.v_q * 4 / 16 * 16;
             size_t lo = (row_bytes / gridDim.x * blockIdx.x) / 16 * 16;
             size_t hi = blockIdx.x + 1 == gridDim.x ? row_bytes : (row_bytes / gridDim.x * (blockIdx.x + 1)) / 16 * 16;
@@ -385,31 +432,87 @@ od_sample_kernel(const SampleArgs a)
     const int ntiles = a.ntiles;
     double *tile_val = a.tile_val + (size_t)b * ntiles;
 
-    // ---- pass 1: the value of every tile ----
-    {
-        const int t_lo = (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
-        int t_hi = t_lo + a.tiles_per_warp;
-        if (t_hi > ntiles) t_hi = ntiles;
-        if (t_lo < t_hi) warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
+    if (MODE != 2) {
+        // ---- pass 1: the value of every tile ----
+        {
+            const int t_lo = tile_lo + (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
+            int t_hi = t_lo + a.tiles_per_warp;
+            if (t_hi > tile_hi) t_hi = tile_hi;
+            if (t_lo < t_hi) warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val, dummy);
+        }
+        __threadfence();                               // the tile values are read by another block
+        __syncthreads();
+        if (threadIdx.x == 0) s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
     }
-    __threadfence();                               // the tile values are read by another block
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
 
     // ---- pass 2 (one block per sequence) ----
     bool residual = q.residual;
     uint32_t flags = residual ? 0u : OD_SF_BONUS;
-    const float u = od_uniform(a.seed[b], a.step, (uint32_t)j, 1u);
-    const int per = (ntiles + OD_SAMPLE_THREADS - 1) / OD_SAMPLE_THREADS;
-    const int my_lo = threadIdx.x * per;
-    const int my_hi = my_lo + per < ntiles ? my_lo + per : ntiles;
+    const float u = MODE == 1 ? 0.f : od_uniform(a.seed[b], a.step, (uint32_t)j, 1u);
+    const int per = (tile_hi - tile_lo + OD_SAMPLE_THREADS - 1) / OD_SAMPLE_THREADS;
+    const int my_lo = tile_lo + threadIdx.x * per < tile_hi ? tile_lo + threadIdx.x * per : tile_hi;
+    const int my_hi = my_lo + per < tile_hi ? my_lo + per : tile_hi;
     // tile values (rounding can leave a tile without residual mass slightly negative)
-    for (int t = threadIdx.x; t < ntiles; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, __ldcg(tile_val + t));
-    if (threadIdx.x == 0) a.ticket[b] = 0;
+    for (int t = tile_lo + threadIdx.x; t < tile_hi; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, __ldcg(tile_val + t));
+    if (MODE != 2 && threadIdx.x == 0) a.ticket[b] = 0;
     __syncthreads();
+
+    if (MODE == 1) {
+        // ---- this shard's shares ----
+        const double mass_r = block_total(s_val, my_lo, my_hi, s_warp);
+        double mass_e = 0.0;
+        if (residual && !(mass_r > 0.0)) {
+            // no residual mass here: should no shard have any, the draw is from p_j
+            for (int t_lo = tile_lo + warp * 4; t_lo < tile_hi; t_lo += WARPS * 4)
+                warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 4 < tile_hi ? t_lo + 4 : tile_hi, lane, tile_val, dummy);
+            __syncthreads();
+            for (int t = tile_lo + threadIdx.x; t < tile_hi; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, tile_val[t]);
+            __syncthreads();
+            mass_e = block_total(s_val, my_lo, my_hi, s_warp);
+        }
+        if (threadIdx.x == 0) { a.mass_out[2 * b] = mass_r; a.mass_out[2 * b + 1] = mass_e; }
+        return;
+    }
+
+    double shard_before = 0.0, shard_total = 0.0;      // MODE 2: sums over the shards before this one / all
+    if (MODE == 2) {
+        double tot_r = 0.0, tot_e = 0.0;
+        for (int s = 0; s < a.n_shards; ++s) {
+            tot_r += a.mass_all[((size_t)s * a.B + b) * 2];
+            tot_e += a.mass_all[((size_t)s * a.B + b) * 2 + 1];
+        }
+        const bool use_e = residual && !(tot_r > 0.0);
+        if (use_e) { residual = false; flags |= OD_SF_ZERO_MASS; }   // the tile values then hold p_j's
+        shard_total = use_e ? tot_e : tot_r;
+        // the shard in which the running sum crosses the target (else the last one with mass)
+        int owner = -1;
+        if (shard_total > 0.0) {
+            const double target = (double)u * shard_total;
+            double c = 0.0;
+            int last = -1;
+            for (int s = 0; s < a.n_shards; ++s) {
+                const double v = a.mass_all[((size_t)s * a.B + b) * 2 + (use_e ? 1 : 0)];
+                if (s == a.shard_index) shard_before = c;
+                if (v > 0.0) last = s;
+                if (c + v > target) { owner = s; break; }
+                c += v;
+            }
+            if (owner < 0) owner = last;
+        }
+        if (owner != a.shard_index) {
+            if (threadIdx.x == 0) {
+                const bool report = owner < 0 && a.shard_index == 0;   // no mass anywhere: shard 0 says so
+                a.out_token[b] = -1;
+                a.resid_mass[b] = report ? (float)(shard_total / (double)q.S) : 0.f;
+                a.flags[b] = report ? (flags | OD_SF_ZERO_MASS) : 0u;
+            }
+            return;
+        }
+    }
+
     for (int attempt = 0; attempt < 2; ++attempt) {
         // exclusive scan of the tile values: thread i owns `per` consecutive tiles
         double loc = 0.0;
@@ -423,11 +526,11 @@ od_sample_kernel(const SampleArgs a)
         if (lane == 31) s_warp[warp] = inc;
         if (threadIdx.x == 0) { s_tile = 0x7FFFFFFF; s_lastmass = -1; s_token = -2; }
         __syncthreads();
-        double base = 0.0;
+        double base = MODE == 2 ? shard_before : 0.0;
         for (int w = 0; w < warp; ++w) base += s_warp[w];
         if (threadIdx.x == OD_SAMPLE_THREADS - 1) s_total = base + inc;
         __syncthreads();
-        const double Rn = s_total;                  // unnormalised total
+        const double Rn = MODE == 2 ? shard_total : s_total;   // unnormalised total
         double target = 0.0;
         if (Rn > 0.0) {
             target = (double)u * Rn;
@@ -500,23 +603,93 @@ od_sample_kernel(const SampleArgs a)
         }
         __syncthreads();
         if (s_token >= 0) return;
-        if (!residual || attempt == 1) break;
+        if (MODE == 2 || !residual || attempt == 1) break;
         // no usable residual mass: draw from p_j instead (rare; this block redoes the row)
         residual = false;
         flags |= OD_SF_ZERO_MASS;
         for (int t_lo = warp * 4; t_lo < ntiles; t_lo += WARPS * 4)
-            warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 4 < ntiles ? t_lo + 4 : ntiles, lane, tile_val);
+            warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 4 < ntiles ? t_lo + 4 : ntiles, lane, tile_val, dummy);
         __syncthreads();
         for (int t = threadIdx.x; t < ntiles; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, tile_val[t]);
         __syncthreads();
     }
     if (threadIdx.x == 0) {                         // no mass at all (non-finite input)
-        a.out_token[b] = -1; a.resid_mass[b] = (float)(s_total / (double)q.S);
+        a.out_token[b] = -1;
+        a.resid_mass[b] = (float)((MODE == 2 ? shard_total : s_total) / (double)q.S);
         a.flags[b] = flags | OD_SF_ZERO_MASS;
     }
 }
 
 }  // namespace
+
+// mode 0: od_sample_residual; 1 / 2: the two calls of a vocabulary shard
+static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, const void *logits,
+                                 int32_t dtype, int64_t row_stride, int64_t seq_stride,
+                                 const float *row_max, const float *row_sum, const float *q_rows,
+                                 const int32_t *draft_ids, const int32_t *tgt_ids,
+                                 const float *q_prime, const int32_t *span_start,
+                                 const int32_t *span_len, const int32_t *m,
+                                 const uint8_t *tail_kind, const int32_t *n_accepted,
+                                 const float *temperature, const uint64_t *seed, uint64_t step,
+                                 int32_t *out_token, float *resid_mass, uint32_t *flags,
+                                 int32_t shard_lo, int32_t shard_len, int32_t n_shards, int32_t shard_index,
+                                 const double *mass_all, double *mass_out, cudaStream_t s)
+{
+    if (B == 0) return cudaSuccess;
+    const int ntiles = c->tiles_per_row;
+    const int tile_lo = mode == 0 ? 0 : shard_lo / OD_SAMPLE_TILE;
+    const int tile_hi = mode == 0 ? ntiles : (shard_lo + shard_len + OD_SAMPLE_TILE - 1) / OD_SAMPLE_TILE;
+    const int wtiles = tile_hi - tile_lo;
+    int64_t tpw = c->opt_sample_tiles_per_warp;
+    if (tpw <= 0) {
+        // one resident wave (four 256-thread blocks per SM) over the whole batch
+        const int64_t want = (int64_t)c->sm_count * 4;
+        int64_t per_row = want / B;
+        if (per_row < 1) per_row = 1;
+        tpw = (wtiles + per_row * WARPS - 1) / (per_row * WARPS);
+        if (tpw < 1) tpw = 1;
+    }
+    const int64_t tiles_per_block = tpw * WARPS;
+    const int blocks_x = mode == 2 ? 1 : (int)((wtiles + tiles_per_block - 1) / tiles_per_block);
+    SampleArgs a = {};
+    a.logits = logits; a.row_stride = row_stride; a.seq_stride = seq_stride;
+    a.B = B; a.K_max = K_max; a.v_p = mode == 0 ? c->v_p : shard_lo + shard_len; a.v_q = c->v_q;
+    a.ntiles = ntiles; a.tiles_per_warp = (int32_t)tpw;
+    a.row_max = row_max; a.row_sum = row_sum; a.q_rows = q_rows;
+    a.draft_ids = draft_ids; a.tgt_ids = tgt_ids; a.q_prime = q_prime;
+    a.span_start = span_start; a.span_len = span_len; a.m = m; a.tail_kind = tail_kind;
+    a.n_accepted = n_accepted; a.temperature = temperature; a.seed = seed; a.step = step;
+    a.vocab_map = c->d_vocab_map; a.inv_map = c->d_inv_map;
+    a.out_token = out_token; a.resid_mass = resid_mass; a.flags = flags;
+    a.tile_val = c->d_tile_sums; a.ticket = c->d_samp_ticket;
+    a.mapped_t = c->d_mapped_t; a.mapped_d = c->d_mapped_d; a.list_width = c->list_width;
+    a.tile_lo = tile_lo; a.tile_hi = tile_hi; a.col0 = mode == 0 ? 0 : shard_lo;
+    a.n_shards = n_shards; a.shard_index = shard_index; a.mass_all = mass_all; a.mass_out = mass_out;
+    if (mode != 2) {
+        c->info[2] = (int64_t)blocks_x * B;
+        c->info[3] = tpw;
+    }
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks_x, (unsigned)B);
+    cfg.blockDim = dim3(OD_SAMPLE_THREADS);
+    cfg.dynamicSmemBytes = (size_t)ntiles * 8;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->opt_pdl ? 1 : 0;
+    const bool bf = dtype == OD_BF16;
+    if (mode == 0)
+        return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 0>, a)
+                  : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 0>, a);
+    if (mode == 1)
+        return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 1>, a)
+                  : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 1>, a);
+    return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 2>, a)
+              : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 2>, a);
+}
 
 cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
                              int32_t dtype, int64_t row_stride, int64_t seq_stride,
@@ -529,44 +702,39 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
                              cudaStream_t s)
 {
-    if (B == 0) return cudaSuccess;
-    const int ntiles = c->tiles_per_row;
-    int64_t tpw = c->opt_sample_tiles_per_warp;
-    if (tpw <= 0) {
-        // one resident wave (four 256-thread blocks per SM) over the whole batch
-        const int64_t want = (int64_t)c->sm_count * 4;
-        int64_t per_row = want / B;
-        if (per_row < 1) per_row = 1;
-        tpw = (ntiles + per_row * WARPS - 1) / (per_row * WARPS);
-        if (tpw < 1) tpw = 1;
-    }
-    const int64_t tiles_per_block = tpw * WARPS;
-    const int blocks_x = (int)((ntiles + tiles_per_block - 1) / tiles_per_block);
-    SampleArgs a;
-    a.logits = logits; a.row_stride = row_stride; a.seq_stride = seq_stride;
-    a.B = B; a.K_max = K_max; a.v_p = c->v_p; a.v_q = c->v_q;
-    a.ntiles = ntiles; a.tiles_per_warp = (int32_t)tpw;
-    a.row_max = row_max; a.row_sum = row_sum; a.q_rows = q_rows;
-    a.draft_ids = draft_ids; a.tgt_ids = tgt_ids; a.q_prime = q_prime;
-    a.span_start = span_start; a.span_len = span_len; a.m = m; a.tail_kind = tail_kind;
-    a.n_accepted = n_accepted; a.temperature = temperature; a.seed = seed; a.step = step;
-    a.vocab_map = c->d_vocab_map; a.inv_map = c->d_inv_map;
-    a.out_token = out_token; a.resid_mass = resid_mass; a.flags = flags;
-    a.tile_val = c->d_tile_sums; a.ticket = c->d_samp_ticket;
-    a.mapped_t = c->d_mapped_t; a.mapped_d = c->d_mapped_d; a.list_width = c->list_width;
-    c->info[2] = (int64_t)blocks_x * B;
-    c->info[3] = tpw;
+    return launch_sample(c, 0, B, K_max, logits, dtype, row_stride, seq_stride, row_max, row_sum, q_rows,
+                         draft_ids, tgt_ids, q_prime, span_start, span_len, m, tail_kind, n_accepted,
+                         temperature, seed, step, out_token, resid_mass, flags, 0, 0, 1, 0, nullptr, nullptr, s);
+}
 
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)blocks_x, (unsigned)B);
-    cfg.blockDim = dim3(OD_SAMPLE_THREADS);
-    cfg.dynamicSmemBytes = (size_t)ntiles * 8;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = c->opt_pdl ? 1 : 0;
-    return dtype == OD_BF16 ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16>, a)
-                            : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32>, a);
+cudaError_t od_launch_sample_shard_mass(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo,
+                                        int32_t shard_len, const void *logits, int32_t dtype,
+                                        int64_t row_stride, int64_t seq_stride, const float *row_max,
+                                        const float *row_sum, const float *q_rows, const int32_t *draft_ids,
+                                        const int32_t *tgt_ids, const float *q_prime,
+                                        const int32_t *span_start, const int32_t *span_len, const int32_t *m,
+                                        const uint8_t *tail_kind, const int32_t *n_accepted,
+                                        const float *temperature, double *mass, cudaStream_t s)
+{
+    return launch_sample(c, 1, B, K_max, logits, dtype, row_stride, seq_stride, row_max, row_sum, q_rows,
+                         draft_ids, tgt_ids, q_prime, span_start, span_len, m, tail_kind, n_accepted,
+                         temperature, nullptr, 0, nullptr, nullptr, nullptr, shard_lo, shard_len, 1, 0,
+                         nullptr, mass, s);
+}
+
+cudaError_t od_launch_sample_shard_pick(od_ctx *c, int32_t B, int32_t K_max, int32_t n_shards,
+                                        int32_t shard_index, int32_t shard_lo, int32_t shard_len,
+                                        const double *mass_all, const void *logits, int32_t dtype,
+                                        int64_t row_stride, int64_t seq_stride, const float *row_max,
+                                        const float *row_sum, const float *q_rows, const int32_t *draft_ids,
+                                        const int32_t *tgt_ids, const float *q_prime,
+                                        const int32_t *span_start, const int32_t *span_len, const int32_t *m,
+                                        const uint8_t *tail_kind, const int32_t *n_accepted,
+                                        const float *temperature, const uint64_t *seed, uint64_t step,
+                                        int32_t *out_token, float *resid_mass, uint32_t *flags, cudaStream_t s)
+{
+    return launch_sample(c, 2, B, K_max, logits, dtype, row_stride, seq_stride, row_max, row_sum, q_rows,
+                         draft_ids, tgt_ids, q_prime, span_start, span_len, m, tail_kind, n_accepted,
+                         temperature, seed, step, out_token, resid_mass, flags, shard_lo, shard_len, n_shards,
+                         shard_index, mass_all, nullptr, s);
 }

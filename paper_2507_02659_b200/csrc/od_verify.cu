@@ -36,6 +36,13 @@
 // end as S_c * exp2(fma(-M, s, c)), which removes the rounding of c. M itself
 // is tracked separately (packed bf16x2 maxima for bf16 rows). The reduction
 // order is fixed by (m, grid): results are bit-identical from run to run.
+//
+// Vocabulary-sharded variant (the target's output layer split by columns over
+// several GPUs): a shard streams its own columns with the same stream kernel,
+// od_verify_shard_stats_kernel folds the partials of a row into one record
+// (c, sum, max, x[t_i] if the shard owns t_i), the records of all shards are
+// exchanged by the caller, and od_verify_finish_kernel merges them (the same
+// pair algebra) and takes the decisions of the decide kernel.
 #include <float.h>
 
 #include "od_common.cuh"
@@ -73,6 +80,12 @@ struct VerifyArgs {
     int32_t *n_accepted, *n_draft_accepted;
     uint32_t *flags;
     float4 *partials;                   // [row slot][OD_VERIFY_SEG_MAX] (c, sum, max, -)
+    // vocabulary shards: v_p above is then the number of columns of this shard
+    int32_t col0;                       // target id of the shard's first column
+    int32_t n_shards;
+    float4 *stats;                      // [row slot] (c, sum, max, x[t_i] or -inf) of this shard
+    const float4 *stats_all;            // [n_shards][rows][4], rows = batch * (K_max + 1)
+    int64_t stats_rows;
 };
 
 // How many blocks hold pieces of flat row `rho` of a space whose blocks take
@@ -419,8 +432,52 @@ od_verify_stream_kernel(const VerifyArgs a)
     }
 }
 
+// Row r of sequence b from its merged statistics (c, s, mx): row maximum and sum,
+// p(t_i), the ratio and the accept / boundary bits (one thread per row).
+__device__ __forceinline__ void decide_row(const VerifyArgs &a, int b, int r, int mb, float c, float s, float mx,
+                                           float scale, bool t_ok, float x_t, float q, float u,
+                                           unsigned int *s_bits)
+{
+    const int row_slot = b * (a.K_max + 1) + r;
+    const float M = mx;
+    const float S = s * od_ex2(fmaf(-M, scale, c));     // sum of exp2((x - M)*scale)
+    a.row_max[row_slot] = M;
+    a.row_sum[row_slot] = S;
+    if (!(S > 0.f) || !(S <= FLT_MAX)) atomicOr(&s_bits[1], 1u);   // not finite and positive
+    if (r < mb) {
+        const size_t o = (size_t)b * a.K_max + r;
+        const float p = t_ok ? od_ex2((x_t - M) * scale) / S : 0.f;
+        const float ra = (q <= p) ? 1.f : p / q;
+        a.p_sel[o] = p;
+        a.ratio[o] = ra;
+        unsigned int bits = 0;
+        if (u < ra) bits |= 1u << r;
+        if (fabsf(u - ra) <= OD_TAU_ACCEPT) bits |= 1u << (16 + r);
+        if (bits) atomicOr(&s_bits[0], bits);
+    }
+}
+
+// The accepted prefix of sequence b from the rows' bits (one thread).
+__device__ __forceinline__ void decide_prefix(const VerifyArgs &a, int b, int mb, bool bad_T,
+                                              const unsigned int *s_bits)
+{
+    const unsigned int all = s_bits[0];
+    int n = 0;
+    while (n < mb && (all >> n & 1u)) ++n;
+    int nd = 0;
+    for (int k = 0; k < n; ++k) nd += a.span_len[(size_t)b * a.K_max + k];
+    uint32_t f = (all >> 16) & OD_VF_BOUNDARY_MASK;
+    if (s_bits[1] & 1u) f |= OD_VF_NONFINITE;
+    if (bad_T) { f |= OD_VF_BAD_TEMPERATURE; n = 0; nd = 0; }
+    a.n_accepted[b] = n;
+    a.n_draft_accepted[b] = nd;
+    a.flags[b] = f;
+}
+
 // One block per sequence, warp r = row r (blockDim = 32 * (K_max + 1)).
-template <int DTYPE>
+// SHARD: the rows are the columns [col0, col0 + v_p) of the full rows; the merged
+// statistics of a row are stored as this shard's record and nothing is decided.
+template <int DTYPE, bool SHARD>
 __global__ void __launch_bounds__(32 * (OD_MAX_K + 1))
 od_verify_decide_kernel(const VerifyArgs a)
 {
@@ -457,11 +514,13 @@ od_verify_decide_kernel(const VerifyArgs a)
     bool t_ok = false;
     if (lane == 0 && r < mb) {
         const size_t o = (size_t)b * a.K_max + r;
-        const int32_t t = a.tgt_ids[o];
+        const int32_t t = a.tgt_ids[o] - (SHARD ? a.col0 : 0);
         t_ok = t >= 0 && t < a.v_p;
         if (t_ok) x_t = od_load_logit<DTYPE>(row, t);
-        q = a.q_prime[o];
-        u = od_uniform(a.seed[b], a.step, (uint32_t)r, 0u);
+        if (!SHARD) {
+            q = a.q_prime[o];
+            u = od_uniform(a.seed[b], a.step, (uint32_t)r, 0u);
+        }
     }
     __syncthreads();
     before = 0; total = 0;
@@ -488,39 +547,59 @@ od_verify_decide_kernel(const VerifyArgs a)
             mx = fmaxf(mx, p.z);
         }
         warp_merge(c, s, mx);
-        if (lane == 0) {
-            const float M = mx;
-            const float S = s * od_ex2(fmaf(-M, scale, c));     // sum of exp2((x - M)*scale)
-            a.row_max[row_slot] = M;
-            a.row_sum[row_slot] = S;
-            if (!(S > 0.f) || !(S <= FLT_MAX)) atomicOr(&s_bits[1], 1u);   // not finite and positive
-            if (r < mb) {
-                const size_t o = (size_t)b * a.K_max + r;
-                const float p = t_ok ? od_ex2((x_t - M) * scale) / S : 0.f;
-                const float ra = (q <= p) ? 1.f : p / q;
-                a.p_sel[o] = p;
-                a.ratio[o] = ra;
-                unsigned int bits = 0;
-                if (u < ra) bits |= 1u << r;
-                if (fabsf(u - ra) <= OD_TAU_ACCEPT) bits |= 1u << (16 + r);
-                if (bits) atomicOr(&s_bits[0], bits);
-            }
+        if (SHARD) {
+            if (lane == 0) a.stats[row_slot] = make_float4(c, s, mx, t_ok ? x_t : -INFINITY);
+        } else {
+            if (lane == 0) decide_row(a, b, r, mb, c, s, mx, scale, t_ok, x_t, q, u, s_bits);
         }
     }
+    if (SHARD) return;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int all = s_bits[0];
-        int n = 0;
-        while (n < mb && (all >> n & 1u)) ++n;
-        int nd = 0;
-        for (int k = 0; k < n; ++k) nd += a.span_len[(size_t)b * a.K_max + k];
-        uint32_t f = (all >> 16) & OD_VF_BOUNDARY_MASK;
-        if (s_bits[1] & 1u) f |= OD_VF_NONFINITE;
-        if (bad_T) { f |= OD_VF_BAD_TEMPERATURE; n = 0; nd = 0; }
-        a.n_accepted[b] = n;
-        a.n_draft_accepted[b] = nd;
-        a.flags[b] = f;
+    if (threadIdx.x == 0) decide_prefix(a, b, mb, bad_T, s_bits);
+}
+
+// Vocabulary shards, after the exchange: one block per sequence, warp r = row r merges
+// the row's records of all shards (in shard order) and decides as above. x[t_i] is the
+// one finite entry among the records (the shard that owns t_i), or -inf.
+__global__ void __launch_bounds__(32 * (OD_MAX_K + 1))
+od_verify_finish_kernel(const VerifyArgs a)
+{
+    __shared__ unsigned int s_bits[2];
+    const int b = blockIdx.x;
+    const int lane = threadIdx.x & 31, r = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { s_bits[0] = 0; s_bits[1] = 0; }
+    const int mb = clamp_m(a.m[b], a.K_max);
+    const float T = a.temperature[b];
+    const bool bad_T = !(T > 0.f);
+    const float scale = bad_T ? 0.f : 1.4426950408889634f / T;
+    float q = 0.f, u = 0.f;
+    bool t_ok = false;
+    if (lane == 0 && r < mb) {
+        const size_t o = (size_t)b * a.K_max + r;
+        const int32_t t = a.tgt_ids[o];
+        t_ok = t >= 0 && t < a.v_p;
+        q = a.q_prime[o];
+        u = od_uniform(a.seed[b], a.step, (uint32_t)r, 0u);
     }
+    __syncthreads();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+    if (r <= mb) {
+        const int row_slot = b * (a.K_max + 1) + r;
+        float c = -FLT_MAX, s = 0.f, mx = -INFINITY, x_t = -INFINITY;
+        for (int k = lane; k < a.n_shards; k += 32) {
+            const float4 p = __ldcg(a.stats_all + (size_t)k * a.stats_rows + row_slot);
+            pair_merge(c, s, p.x, p.y);
+            mx = fmaxf(mx, p.z);
+            x_t = fmaxf(x_t, p.w);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) x_t = fmaxf(x_t, __shfl_xor_sync(0xFFFFFFFFu, x_t, off));
+        warp_merge(c, s, mx);
+        if (lane == 0) decide_row(a, b, r, mb, c, s, mx, scale, t_ok, x_t, q, u, s_bits);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) decide_prefix(a, b, mb, bad_T, s_bits);
 }
 
 template <typename Kern>
@@ -540,6 +619,41 @@ cudaError_t launch(Kern kern, unsigned grid, unsigned block, cudaStream_t s, boo
 
 }  // namespace
 
+// Launch plan of the stream kernel for `nb` sequences whose rows hold `v_len` elements.
+static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_len, int32_t dtype, VerifyArgs &a)
+{
+    const int64_t esz = dtype == OD_BF16 ? 2 : 4;
+    const int64_t row_bytes = (int64_t)v_len * esz;
+    const int32_t W = (int32_t)((row_bytes + 511) / 512);
+    // a row is cut into at most OD_VERIFY_SEG_MAX / WARPS block segments (one partial per warp each)
+    constexpr int MAX_BLOCK_SEGS = OD_VERIFY_SEG_MAX / WARPS;
+    const int32_t span_min = (W + MAX_BLOCK_SEGS - 2) / (MAX_BLOCK_SEGS - 1);
+    int64_t blocks_per_sm = c->opt_verify_blocks_per_sm > 0 ? c->opt_verify_blocks_per_sm : OD_VERIFY_BLOCKS_PER_SM;
+    if (blocks_per_sm > OD_VERIFY_BLOCKS_PER_SM) blocks_per_sm = OD_VERIFY_BLOCKS_PER_SM;
+    // no more blocks than the most this slice can need
+    const int64_t max_units = (int64_t)nb * (K_max + 1) * W;
+    int64_t grid = (int64_t)c->sm_count * blocks_per_sm * (c->opt_verify_waves > 0 ? c->opt_verify_waves : 1);
+    const int64_t need = max_units / span_min + 1;
+    if (grid > need) grid = need;
+    if (grid < 1) grid = 1;
+    a.B = nb; a.K_max = K_max; a.v_p = v_len;
+    a.W = W; a.n_chunks = (int32_t)grid; a.span_min = span_min;
+    int64_t span_a = ((int64_t)nb * W + grid - 1) / grid;
+    if (span_a < span_min) span_a = span_min;
+    a.span_a = (int32_t)span_a;
+    a.a_early = span_a / W + 2 <= A_PARK;
+}
+
+// batches beyond the shared-memory prefix table go in slices; a slice's flat
+// unit indices (plus one span of slack) must fit 32 bits
+static int32_t slice_of(int32_t K_max, int32_t v_len, int32_t dtype)
+{
+    const int64_t W = ((int64_t)v_len * (dtype == OD_BF16 ? 2 : 4) + 511) / 512;
+    int32_t slice = OD_VERIFY_MAX_B;
+    while (slice > 1 && (int64_t)slice * (K_max + 1) * W > (int64_t)1 << 30) slice >>= 1;
+    return slice;
+}
+
 cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
                              int32_t dtype, int64_t row_stride, int64_t seq_stride,
                              const int32_t *tgt_ids, const float *q_prime,
@@ -550,35 +664,13 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              uint32_t *flags, cudaStream_t s)
 {
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
-    const int64_t row_bytes = (int64_t)c->v_p * esz;
-    const int32_t W = (int32_t)((row_bytes + 511) / 512);
-    // a row is cut into at most OD_VERIFY_SEG_MAX / WARPS block segments (one partial per warp each)
-    constexpr int MAX_BLOCK_SEGS = OD_VERIFY_SEG_MAX / WARPS;
-    const int32_t span_min = (W + MAX_BLOCK_SEGS - 2) / (MAX_BLOCK_SEGS - 1);
-    int64_t blocks_per_sm = c->opt_verify_blocks_per_sm > 0 ? c->opt_verify_blocks_per_sm : OD_VERIFY_BLOCKS_PER_SM;
-    if (blocks_per_sm > OD_VERIFY_BLOCKS_PER_SM) blocks_per_sm = OD_VERIFY_BLOCKS_PER_SM;
-
-    // batches beyond the shared-memory prefix table go in slices; a slice's flat
-    // unit indices (plus one span of slack) must fit 32 bits
-    int32_t slice = OD_VERIFY_MAX_B;
-    while (slice > 1 && (int64_t)slice * (K_max + 1) * W > (int64_t)1 << 30) slice >>= 1;
+    const int32_t slice = slice_of(K_max, c->v_p, dtype);
     for (int32_t b0 = 0; b0 < B; b0 += slice) {
         const int32_t nb = B - b0 < slice ? B - b0 : slice;
-        // no more blocks than the most this slice can need
-        const int64_t max_units = (int64_t)nb * (K_max + 1) * W;
-        int64_t grid = (int64_t)c->sm_count * blocks_per_sm * (c->opt_verify_waves > 0 ? c->opt_verify_waves : 1);
-        const int64_t need = max_units / span_min + 1;
-        if (grid > need) grid = need;
-        if (grid < 1) grid = 1;
-        VerifyArgs a;
+        VerifyArgs a = {};
+        plan_stream(c, nb, K_max, c->v_p, dtype, a);
         a.logits = (const char *)logits + (size_t)b0 * seq_stride * esz;
         a.row_stride = row_stride; a.seq_stride = seq_stride;
-        a.B = nb; a.K_max = K_max; a.v_p = c->v_p;
-        a.W = W; a.n_chunks = (int32_t)grid; a.span_min = span_min;
-        int64_t span_a = ((int64_t)nb * W + grid - 1) / grid;
-        if (span_a < span_min) span_a = span_min;
-        a.span_a = (int32_t)span_a;
-        a.a_early = span_a / W + 2 <= A_PARK;
         a.tgt_ids = tgt_ids + (size_t)b0 * K_max; a.q_prime = q_prime + (size_t)b0 * K_max;
         a.span_len = span_len + (size_t)b0 * K_max; a.m = m + b0;
         a.temperature = temperature + b0; a.seed = seed + b0; a.step = step;
@@ -587,19 +679,78 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
         a.n_accepted = n_accepted + b0; a.n_draft_accepted = n_draft_accepted + b0;
         a.flags = flags + b0;
         a.partials = c->d_partials;
-        c->info[0] = grid;
-        c->info[1] = span_a;
+        c->info[0] = a.n_chunks;
+        c->info[1] = a.span_a;
 
         const bool pdl = c->opt_pdl != 0;
         cudaError_t e = dtype == OD_BF16
-            ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)grid, THREADS, s, pdl, a)
-            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)grid, THREADS, s, pdl, a);
+            ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)a.n_chunks, THREADS, s, pdl, a)
+            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)a.n_chunks, THREADS, s, pdl, a);
         if (e != cudaSuccess) return e;
         const unsigned dthreads = 32u * (unsigned)(K_max + 1);
         e = dtype == OD_BF16
-            ? launch(od_verify_decide_kernel<OD_BF16>, (unsigned)nb, dthreads, s, pdl, a)
-            : launch(od_verify_decide_kernel<OD_F32>, (unsigned)nb, dthreads, s, pdl, a);
+            ? launch(od_verify_decide_kernel<OD_BF16, false>, (unsigned)nb, dthreads, s, pdl, a)
+            : launch(od_verify_decide_kernel<OD_F32, false>, (unsigned)nb, dthreads, s, pdl, a);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+// One vocabulary shard: the statistics of columns [shard_lo, shard_lo + shard_len) of
+// every row, one record per row into stats[B * (K_max + 1)].
+cudaError_t od_launch_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo,
+                                         int32_t shard_len, const void *logits, int32_t dtype,
+                                         int64_t row_stride, int64_t seq_stride, const int32_t *tgt_ids,
+                                         const int32_t *m, const float *temperature, float *stats,
+                                         cudaStream_t s)
+{
+    const int64_t esz = dtype == OD_BF16 ? 2 : 4;
+    const int32_t slice = slice_of(K_max, shard_len, dtype);
+    for (int32_t b0 = 0; b0 < B; b0 += slice) {
+        const int32_t nb = B - b0 < slice ? B - b0 : slice;
+        VerifyArgs a = {};
+        plan_stream(c, nb, K_max, shard_len, dtype, a);
+        a.logits = (const char *)logits + (size_t)b0 * seq_stride * esz;
+        a.row_stride = row_stride; a.seq_stride = seq_stride;
+        a.tgt_ids = tgt_ids + (size_t)b0 * K_max; a.m = m + b0;
+        a.temperature = temperature + b0;
+        a.partials = c->d_partials;
+        a.col0 = shard_lo;
+        a.stats = (float4 *)stats + (size_t)b0 * (K_max + 1);
+        c->info[0] = a.n_chunks;
+        c->info[1] = a.span_a;
+        const bool pdl = c->opt_pdl != 0;
+        cudaError_t e = dtype == OD_BF16
+            ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)a.n_chunks, THREADS, s, pdl, a)
+            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)a.n_chunks, THREADS, s, pdl, a);
+        if (e != cudaSuccess) return e;
+        const unsigned dthreads = 32u * (unsigned)(K_max + 1);
+        e = dtype == OD_BF16
+            ? launch(od_verify_decide_kernel<OD_BF16, true>, (unsigned)nb, dthreads, s, pdl, a)
+            : launch(od_verify_decide_kernel<OD_F32, true>, (unsigned)nb, dthreads, s, pdl, a);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// After the exchange: merge the records of all shards and decide.
+cudaError_t od_launch_verify_shard_finish(od_ctx *c, int32_t B, int32_t K_max, int32_t n_shards,
+                                          const float *stats_all, const int32_t *tgt_ids,
+                                          const float *q_prime, const int32_t *span_len, const int32_t *m,
+                                          const float *temperature, const uint64_t *seed, uint64_t step,
+                                          float *row_max, float *row_sum, float *p_sel, float *ratio,
+                                          int32_t *n_accepted, int32_t *n_draft_accepted, uint32_t *flags,
+                                          cudaStream_t s)
+{
+    if (B == 0) return cudaSuccess;
+    VerifyArgs a = {};
+    a.B = B; a.K_max = K_max; a.v_p = c->v_p;
+    a.tgt_ids = tgt_ids; a.q_prime = q_prime; a.span_len = span_len; a.m = m;
+    a.temperature = temperature; a.seed = seed; a.step = step;
+    a.row_max = row_max; a.row_sum = row_sum; a.p_sel = p_sel; a.ratio = ratio;
+    a.n_accepted = n_accepted; a.n_draft_accepted = n_draft_accepted; a.flags = flags;
+    a.n_shards = n_shards;
+    a.stats_all = (const float4 *)stats_all;
+    a.stats_rows = (int64_t)B * (K_max + 1);
+    return launch(od_verify_finish_kernel, (unsigned)B, 32u * (unsigned)(K_max + 1), s, c->opt_pdl != 0, a);
 }

@@ -48,7 +48,10 @@ class Workload:
 
 
 def paper_config(i: int) -> Workload:
-    """The five workloads of the benchmark definition (1-based)."""
+    """The five workloads of the benchmark definition (1-based), and as number 6
+    the same-vocabulary setting of the paper's Vicuna-7B experiments (Section 4.2:
+    Llama-68M drafting for a target that shares its 32000-id tokenizer, so the map
+    is the identity and the n-gram cache stays empty) as a larger ragged batch."""
     base = dict(v_q=32000, mapped_frac=0.7, sigma=3.0)
     if i == 1:
         return Workload("cfg1", B=1, steps=1000, k_max=4, k_min=4, v_p=32000,
@@ -80,6 +83,12 @@ def paper_config(i: int) -> Workload:
                         hit_prob=0.2, logit_kind="corr", rho=0.6,
                         temperatures=(1.0,), per_seq_seed=True,
                         gen_seed=0xDA7A0005, **base)
+    if i == 6:
+        return Workload("cfg6", B=256, steps=200, k_max=8, k_min=1, v_p=32000,
+                        logit_dtype="bf16", map_kind="identity", cache_entries=0,
+                        hit_prob=0.0, logit_kind="noise", rho=0.0,
+                        temperatures=(0.7, 1.0), per_seq_seed=True,
+                        gen_seed=0xDA7A0006, **base)
     raise ValueError(f"no such config: {i}")
 
 

@@ -127,6 +127,16 @@ def test_config5_full_batch_sampled_sequences(cuda_device):
     _assert_rates(s)
 
 
+def test_same_vocabulary_ragged_batch_sampled_sequences(cuda_device):
+    """Workload 6: 256 sequences, identity map over 32000 ids, no cache, ragged K."""
+    w = synth.paper_config(6)
+    sel = np.arange(0, 256, 3)
+    s = _run_workload(w, cuda_device, [0, 1], sel=sel)
+    assert s.sequences == 2 * len(sel)
+    assert s.cache_hits == 0 and s.unmapped_stops == 0
+    _assert_rates(s)
+
+
 # ------------------------------------------------------------ properties
 def test_results_are_bit_identical_run_to_run(cuda_device):
     w = _small("det", B=48, v_q=3000, v_p=50000, cache_entries=1000, gen_seed=0xBEEF60)

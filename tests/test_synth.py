@@ -11,6 +11,8 @@ def test_paper_configs_have_the_published_shapes():
     for i, (B, K, vp, dt, E) in enumerate(shapes, start=1):
         w = synth.paper_config(i)
         assert (w.B, w.k_max, w.v_q, w.v_p, w.logit_dtype, w.cache_entries) == (B, K, 32000, vp, dt, E)
+    w = synth.paper_config(6)      # same vocabulary on both sides: identity map, no cache
+    assert (w.B, w.k_min, w.k_max, w.v_q, w.v_p, w.map_kind, w.cache_entries) == (256, 1, 8, 32000, 32000, "identity", 0)
 
 
 def test_static_is_deterministic_and_well_formed():
