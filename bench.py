@@ -61,6 +61,9 @@ def parse():
                     help="time the online-cache update path (insert + trim) instead of the verification step")
     ap.add_argument("--distill", action="store_true",
                     help="time the distillation loss + gradient (Eq. 3) of the step's proposals instead")
+    ap.add_argument("--vocab-shards", type=int, default=0,
+                    help="time one rank's kernels of the step with the target vocabulary split over this many GPUs")
+    ap.add_argument("--shard-index", type=int, default=-1, help="the shard that is timed (default: the middle one)")
     ap.add_argument("--verify-blocks-per-sm", type=int, default=0)
     ap.add_argument("--verify-waves", type=int, default=0)
     ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
@@ -325,6 +328,110 @@ def run_distill(a):
     ctx.close()
 
 
+def run_vocab_shard(a):
+    """One rank's share of a step whose target vocabulary is split over N GPUs: the
+    five launches groups of that rank (od_map_proposals, od_verify_shard_stats,
+    od_verify_shard_finish, od_sample_shard_mass, od_sample_shard_pick) on its own
+    columns, timed on one GPU. The records of the other shards are computed
+    beforehand and sit in the exchange buffers, so the decisions are those of the
+    real step; the three all-gathers (16 B per row, 16 B and 12 B per sequence) are
+    not part of the number."""
+    from paper_2507_02659_b200 import binding as od
+    from paper_2507_02659_b200 import synth, vshard
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    w = synth.paper_config(a.config)
+    st = synth.make_static(w)
+    N = a.vocab_shards
+    r = a.shard_index if a.shard_index >= 0 else N // 2
+    lo, hi = vshard.split_vocab(w.v_p, r, N)
+    B, K = w.B, w.k_max
+    ctx = od.Context(dev, w.v_q, w.v_p, B, K)
+    ctx.set_vocab_map(st.vocab_map)
+    ctx.cache_build(st.runs, st.run_len, st.run_target)
+    full0 = synth.make_step(w, st, 0, device=dev)
+    esz = full0.logits.element_size()
+    shard_bytes = B * (K + 1) * (hi - lo) * esz
+    P = max(3, -(-4 * L2_BYTES // shard_bytes))
+    P = min(P, 64, a.steps + a.warmup)
+    pool, shard_logits, mps, stats_all, mass_all, vos, sos = [], [], [], [], [], [], []
+    for i in range(P):
+        s = full0 if i == 0 else synth.make_step(w, st, i, device=dev)
+        mp = od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel)
+        bounds = [vshard.split_vocab(w.v_p, k, N) for k in range(N)]
+        sa = torch.stack([od.od_verify_shard_stats(ctx, l, s.logits[:, :, l:h], mp, s.temperature) for l, h in bounds])
+        vo = od.od_verify_shard_finish(ctx, sa, mp, s.temperature, s.seed, i)
+        ma = torch.stack([od.od_sample_shard_mass(ctx, l, s.logits[:, :, l:h], vo, s.q_rows, s.draft_ids, mp,
+                                                  s.temperature) for l, h in bounds])
+        shard_logits.append(s.logits[:, :, lo:hi].contiguous())       # the rank's own dense buffer
+        pool.append(synth.StepInputs(s.draft_ids, s.draft_len, s.q_sel, s.q_rows, shard_logits[-1],
+                                     s.temperature, s.seed, s.step))
+        mps.append(mp); stats_all.append(sa); mass_all.append(ma); vos.append(vo)
+        sos.append(od.alloc_sample_out(ctx, B))
+        del s
+    torch.cuda.synchronize(dev)
+    rows = [int((mps[i].m.clamp(0, K) + 1).sum().item()) for i in range(P)]
+    toks = [int(pool[i].draft_len.sum().item()) for i in range(P)]
+
+    def k1(i):
+        s = pool[i]
+        od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel, out=mps[i])
+
+    def k2(i, step):
+        s = pool[i]
+        od.od_verify_shard_stats(ctx, lo, s.logits, mps[i], s.temperature, out=stats_all[i][r])
+        od.od_verify_shard_finish(ctx, stats_all[i], mps[i], s.temperature, s.seed, i, out=vos[i])
+
+    def k3(i, step):
+        s = pool[i]
+        od.od_sample_shard_mass(ctx, lo, s.logits, vos[i], s.q_rows, s.draft_ids, mps[i], s.temperature,
+                                out=mass_all[i][r])
+        od.od_sample_shard_pick(ctx, r, lo, mass_all[i], s.logits, vos[i], s.q_rows, s.draft_ids, mps[i],
+                                s.temperature, s.seed, i, out=sos[i])
+
+    def full_step(step):
+        i = step % P
+        k1(i); k2(i, step); k3(i, step)
+
+    def graph_ms(fn):
+        for step in range(max(3, a.warmup)):
+            fn(step)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for step in range(a.steps):
+                fn(a.warmup + step)
+        g.replay(); torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); g.replay(); e1.record(); torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / a.steps
+
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    ms_step = graph_ms(full_step)
+    clocks = sampler.stop()
+    ms_k2 = graph_ms(lambda step: k2(step % P, step))
+    ms_k3 = graph_ms(lambda step: k3(step % P, step))
+    row_bytes = (hi - lo) * esz
+    k2_bytes = sum(rows[(a.warmup + k) % P] for k in range(a.steps)) / a.steps * row_bytes
+    tokens = sum(toks[(a.warmup + k) % P] for k in range(a.steps)) / a.steps
+    peak, peak_src = measured_peak()
+    ach = k2_bytes / (ms_k2 * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": a.steps,
+        "warmup": a.warmup, "ms_per_step": ms_step, "higher_is_better": True, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": f"{w.name}, one of {N} vocabulary shards (shard {r}: target ids [{lo}, {hi}))",
+                   "B": B, "k_max": K, "target_vocab": w.v_p, "logit_dtype": w.logit_dtype, "pool_buffers": P,
+                   "l2_policy": f"{P} distinct shard buffers, {P * shard_bytes / 2**20:.0f} MiB of logits cycled",
+                   "exchanges": "not timed: the other shards' records are precomputed in the exchange buffers"},
+        "kernels_ms_per_step": {"od_verify_shard_stats+finish": ms_k2, "od_sample_shard_mass+pick": ms_k3},
+        "roofline": {"kernel": "od_verify_shard_stats + od_verify_shard_finish", "bound": "hbm", "achieved": ach,
+                     "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_source": peak_src,
+                     "bytes_per_launch": k2_bytes, "traffic": None},
+        "gpu_launches": 6 * a.steps, "clocks": clocks}))
+    ctx.close()
+
+
 def main():
     a = parse()
     if a.impl == "reference":
@@ -333,6 +440,8 @@ def main():
         return run_distill(a)
     if a.cache_update:
         return run_cache_update(a)
+    if a.vocab_shards:
+        return run_vocab_shard(a)
     if a.warmup < 3:
         a.warmup = 3
 
