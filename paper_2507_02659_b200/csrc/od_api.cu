@@ -458,6 +458,7 @@ int32_t od_distill_loss(od_ctx *c, int32_t B, int32_t K_max, const float *q_rows
         return OD_ERR_INVALID_ARG;
     DeviceGuard g(c->device);
     if (!g.ok) return OD_ERR_CUDA;
+    c->last_was_map = false;
     OD_CUDA(od_launch_distill(c, B, K_max, q_rows, draft_ids, tgt_ids, span_start, span_len, m, logits,
                               logit_dtype, row_stride, seq_stride, row_max, row_sum, p_sel, temperature,
                               lambda, lambda_mode, loss, grad, (cudaStream_t)stream));
@@ -473,6 +474,7 @@ int32_t od_exit_rule(od_ctx *c, int32_t B, int32_t K_max, const float *head_logi
     if (!(gamma >= 0.f && gamma <= 1.f)) return OD_ERR_INVALID_ARG;
     DeviceGuard g(c->device);
     if (!g.ok) return OD_ERR_CUDA;
+    c->last_was_map = false;
     OD_CUDA(od_launch_exit(B, K_max, head_logits, avail_len, gamma, draft_len, reject_prob, exit_flags,
                            (cudaStream_t)stream));
     return OD_OK;

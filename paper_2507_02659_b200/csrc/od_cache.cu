@@ -310,6 +310,7 @@ int32_t od_cache_insert(od_ctx *c, int32_t N, const int32_t *runs, const int32_t
     Guard g(c->device);
     if (!g.ok) return OD_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
+    c->last_was_map = false;
     const int threads = 128, blocks = (N + threads - 1) / threads;
     insert_claim_kernel<<<blocks, threads, 0, s>>>(N, c->v_q, c->v_p, runs, len, target,
                                                    (unsigned long long *)c->d_keys, c->d_vals, c->cap,
@@ -328,6 +329,7 @@ int32_t od_cache_trim(od_ctx *c, void *stream)
     Guard g(c->device);
     if (!g.ok) return OD_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
+    c->last_was_map = false;
     TrimState *st = (TrimState *)c->d_trim;
     const int grid = c->sm_count * 4;
     trim_begin_kernel<<<1, 1, 0, s>>>(st, (unsigned int)c->dyn_max);

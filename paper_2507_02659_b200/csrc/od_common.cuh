@@ -64,6 +64,10 @@ struct od_ctx {
     int64_t opt_sample_tiles_per_warp;
     int64_t opt_pdl;                // launch with programmatic stream serialization
 
+    // the last launch on this context was the translation kernel, which lets the next
+    // kernel start before its own outputs exist (see od_sample.cu)
+    bool last_was_map;
+
     // last launch info
     int64_t info[4];
 

@@ -170,6 +170,7 @@ cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *dr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = c->opt_pdl ? 1 : 0;
+    c->last_was_map = true;
     return cudaLaunchKernelEx(&cfg, od_map_kernel, B, K_max, c->v_q, draft_ids, draft_len, q_sel,
                               (const int32_t *)c->d_vocab_map, (const uint64_t *)c->d_keys,
                               (const int32_t *)c->d_vals, c->cap, tgt_ids, q_prime, span_start,

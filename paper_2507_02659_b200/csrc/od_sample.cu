@@ -74,6 +74,7 @@ struct SampleArgs {
     int32_t n_shards, shard_index;
     const double *mass_all;             // [n_shards][B][2] (residual share, share of p_j or 0)
     double *mass_out;                   // [B][2] this shard's shares
+    int32_t early;                      // 1: the translation's outputs may be read before griddepcontrol.wait
 };
 
 // what one sequence's warps need to evaluate r(t)
@@ -358,19 +359,43 @@ od_sample_kernel(const SampleArgs a)
     __shared__ int s_tile, s_lastmass, s_token;
     __shared__ double s_before, s_total;
 
-    // n_accepted and the row statistics come from the verification kernels
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;");
-
     const int b = blockIdx.y;
     const int K = a.K_max;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    // Under programmatic dependent launch this grid is resident while the verification
+    // kernels still run. What the translation kernel wrote (it finished before them) is
+    // read now, for every position the step can stop at: lane k of every warp prepares
+    // position k. After the wait only n_accepted and the row statistics are missing.
+    // (a.early = 0: the launch before this one was not od_verify; everything waits.)
+    asm volatile("griddepcontrol.launch_dependents;");
+    if (!a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
     int mb = a.m[b];
     mb = mb < 0 ? 0 : (mb > K ? K : mb);
-    int j = a.n_accepted[b];
-    j = j < 0 ? 0 : (j > mb ? mb : j);
     const bool stop = a.tail_kind[b] == OD_TAIL_UNMAPPED_STOP;
     const float T = a.temperature[b];
+    int32_t e_s0 = 0, e_len = 1, e_tgt = -1, e_d1 = -1, e_pm = -1;
+    float e_qp = 0.f, e_qd1 = 0.f;
+    if (lane < K && lane <= mb) {
+        const size_t o = (size_t)b * K + lane;
+        int s0 = a.span_start[o];
+        e_s0 = s0 < 0 ? 0 : (s0 >= K ? K - 1 : s0);
+        e_len = lane < mb ? a.span_len[o] : 1;
+        if (e_len >= 2) {
+            e_tgt = a.tgt_ids[o];
+            e_qp = a.q_prime[o];
+            const int32_t d1 = a.draft_ids[(size_t)b * K + e_s0];
+            if (d1 >= 0 && d1 < a.v_q) {
+                e_d1 = d1;
+                e_pm = __ldg(a.vocab_map + d1);
+                e_qd1 = __ldg(a.q_rows + ((size_t)b * K + e_s0) * a.v_q + d1);
+            }
+        }
+    }
+
+    // n_accepted and the row statistics come from the verification kernels
+    if (a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
+
     if (!(T > 0.f)) {                              // every block of the sequence leaves here
         if (blockIdx.x == 0 && threadIdx.x == 0) {
             if (MODE == 1) {
@@ -381,6 +406,10 @@ od_sample_kernel(const SampleArgs a)
         }
         return;
     }
+    float rm = 0.f, rs = 0.f;                      // lane k: statistics of row k
+    if (lane <= mb) { rm = a.row_max[b * (K + 1) + lane]; rs = a.row_sum[b * (K + 1) + lane]; }
+    int j = a.n_accepted[b];
+    j = j < 0 ? 0 : (j > mb ? mb : j);
     const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
     // a shard's tiles and ids keep their numbers of the full row: the row pointer is
     // moved back by the shard's first column, and only ids of the window are read
@@ -394,37 +423,40 @@ od_sample_kernel(const SampleArgs a)
     {
         // reference exponent c = fl(M*scale); the rounding of c goes into S exactly:
         // sum_t exp2(x_t*scale - c) = (sum_t exp2((x_t - M)*scale)) * exp2(M*scale - c)
-        const float M = a.row_max[b * (K + 1) + j];
+        const float M = __shfl_sync(0xFFFFFFFFu, rm, j);
         q.c = fmaxf(M * q.scale, -FLT_MAX);
-        q.S = a.row_sum[b * (K + 1) + j] * od_ex2(fmaf(M, q.scale, -q.c));
+        q.S = __shfl_sync(0xFFFFFFFFu, rs, j) * od_ex2(fmaf(M, q.scale, -q.c));
     }
     q.residual = (j < mb) || stop;
     q.ngram_token = -1; q.prefix_token = -1; q.first_draft = -1; q.ngram_prob = 0.f; q.prefix_val = 0.f;
     q.q_row = a.q_rows;
-    if (q.residual) {
-        const size_t o = (size_t)b * K + j;
-        int s0 = a.span_start[o];
-        s0 = s0 < 0 ? 0 : (s0 >= K ? K - 1 : s0);
-        q.q_row = a.q_rows + ((size_t)b * K + s0) * a.v_q;
-        // the gathers of pass 1 come two round trips from now: have the copy engine pull
-        // this block's share of the drafter's row into L2 meanwhile
-        if (MODE != 2 && threadIdx.x == 0) {
-            const size_t row_bytes = (size_t)a.v_q * 4 / 16 * 16;
-            size_t lo = (row_bytes / gridDim.x * blockIdx.x) / 16 * 16;
-            size_t hi = blockIdx.x + 1 == gridDim.x ? row_bytes : (row_bytes / gridDim.x * (blockIdx.x + 1)) / 16 * 16;
-            const char *base = (const char *)q.q_row;
-            if (((uintptr_t)base & 15u) == 0 && hi > lo)
-                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + lo), "r"((uint32_t)(hi - lo)) : "memory");
-        }
-        const int len = j < mb ? a.span_len[o] : 1;
-        if (len >= 2) {
-            q.ngram_token = a.tgt_ids[o];
-            q.ngram_prob = a.q_prime[o];
-            const int32_t d1 = a.draft_ids[(size_t)b * K + s0];
-            if (d1 >= 0 && d1 < a.v_q) {
-                q.first_draft = d1;
-                q.prefix_token = __ldg(a.vocab_map + d1);
-                q.prefix_val = __ldg(q.q_row + d1) - q.ngram_prob;
+    {
+        // position j's preparation (j < K whenever the draw is a residual one)
+        const int src = j < K ? j : 0;
+        const int32_t s0 = __shfl_sync(0xFFFFFFFFu, e_s0, src), len = __shfl_sync(0xFFFFFFFFu, e_len, src);
+        const int32_t tgt = __shfl_sync(0xFFFFFFFFu, e_tgt, src), d1 = __shfl_sync(0xFFFFFFFFu, e_d1, src);
+        const int32_t pm = __shfl_sync(0xFFFFFFFFu, e_pm, src);
+        const float qp = __shfl_sync(0xFFFFFFFFu, e_qp, src), qd1 = __shfl_sync(0xFFFFFFFFu, e_qd1, src);
+        if (q.residual) {
+            q.q_row = a.q_rows + ((size_t)b * K + s0) * a.v_q;
+            // the gathers of pass 1 come two round trips from now: have the copy engine pull
+            // this block's share of the drafter's row into L2 meanwhile
+            if (MODE != 2 && threadIdx.x == 0) {
+                const size_t row_bytes = (size_t)a.v_q * 4 / 16 * 16;
+                size_t lo = (row_bytes / gridDim.x * blockIdx.x) / 16 * 16;
+                size_t hi = blockIdx.x + 1 == gridDim.x ? row_bytes : (row_bytes / gridDim.x * (blockIdx.x + 1)) / 16 * 16;
+                const char *base = (const char *)q.q_row;
+                if (((uintptr_t)base & 15u) == 0 && hi > lo)
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + lo), "r"((uint32_t)(hi - lo)) : "memory");
+            }
+            if (len >= 2) {
+                q.ngram_token = tgt;
+                q.ngram_prob = qp;
+                if (d1 >= 0) {
+                    q.first_draft = d1;
+                    q.prefix_token = pm;
+                    q.prefix_val = qd1 - q.ngram_prob;
+                }
             }
         }
     }
@@ -665,6 +697,10 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     a.mapped_t = c->d_mapped_t; a.mapped_d = c->d_mapped_d; a.list_width = c->list_width;
     a.tile_lo = tile_lo; a.tile_hi = tile_hi; a.col0 = mode == 0 ? 0 : shard_lo;
     a.n_shards = n_shards; a.shard_index = shard_index; a.mass_all = mass_all; a.mass_out = mass_out;
+    // the translation kernel releases its successor before it has written anything: directly
+    // after it, nothing may be read early
+    a.early = c->last_was_map ? 0 : 1;
+    c->last_was_map = false;
     if (mode != 2) {
         c->info[2] = (int64_t)blocks_x * B;
         c->info[3] = tpw;

@@ -485,6 +485,12 @@ od_verify_decide_kernel(const VerifyArgs a)
     __shared__ int32_t s_part[2][OD_MAX_K + 1];
     __shared__ unsigned int s_bits[2];
 
+    // The next kernel of the stream may be placed as soon as this grid is resident: what
+    // it does before its own griddepcontrol.wait (the sampler: nothing; the next step's
+    // stream kernel: row 0 of its sequences) then fills the multiprocessors that the
+    // stream kernel's last blocks leave idle. Its wait still covers this whole grid.
+    asm volatile("griddepcontrol.launch_dependents;");
+
     const int b = blockIdx.x;
     const int lane = threadIdx.x & 31, r = threadIdx.x >> 5;
     const uint32_t W = (uint32_t)a.W;
@@ -535,7 +541,6 @@ od_verify_decide_kernel(const VerifyArgs a)
 
     // ---- the partials
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;");
 
     if (r <= mb) {
         const int row_slot = b * (a.K_max + 1) + r;
@@ -665,6 +670,7 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
 {
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
     const int32_t slice = slice_of(K_max, c->v_p, dtype);
+    c->last_was_map = false;
     for (int32_t b0 = 0; b0 < B; b0 += slice) {
         const int32_t nb = B - b0 < slice ? B - b0 : slice;
         VerifyArgs a = {};
@@ -706,6 +712,7 @@ cudaError_t od_launch_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, in
 {
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
     const int32_t slice = slice_of(K_max, shard_len, dtype);
+    c->last_was_map = false;
     for (int32_t b0 = 0; b0 < B; b0 += slice) {
         const int32_t nb = B - b0 < slice ? B - b0 : slice;
         VerifyArgs a = {};
@@ -742,6 +749,7 @@ cudaError_t od_launch_verify_shard_finish(od_ctx *c, int32_t B, int32_t K_max, i
                                           int32_t *n_accepted, int32_t *n_draft_accepted, uint32_t *flags,
                                           cudaStream_t s)
 {
+    c->last_was_map = false;
     if (B == 0) return cudaSuccess;
     VerifyArgs a = {};
     a.B = B; a.K_max = K_max; a.v_p = c->v_p;

@@ -155,6 +155,27 @@ def test_results_are_bit_identical_run_to_run(cuda_device):
     ctx.close()
 
 
+def test_sampling_directly_after_the_translation_gives_the_same_token(cuda_device):
+    """od_sample_residual prepares its positions before it waits for the kernel in front of it;
+    directly behind od_map_proposals (whose outputs it reads) it must not."""
+    w = _small("mapsample", B=64, v_q=3000, v_p=40000, cache_entries=1000, gen_seed=0xBEEF65)
+    st = synth.make_static(w)
+    ctx = parity.make_context(w, st, cuda_device)
+    s = synth.make_step(w, st, 0, device=cuda_device)
+    mp, vo, so = parity.gpu_step(ctx, s)
+    for _ in range(5):
+        mp2 = od.alloc_map_out(ctx, w.B, w.k_max)
+        for t in (mp2.tgt_ids, mp2.span_start, mp2.span_len, mp2.m):
+            t.fill_(-1)                                  # whatever is read too early is wrong
+        torch.cuda.synchronize()
+        od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel, out=mp2)
+        so2 = od.od_sample_residual(ctx, s.logits, vo, s.q_rows, s.draft_ids, mp2, s.temperature, s.seed, s.step)
+        torch.cuda.synchronize()
+        assert torch.equal(so2.out_token, so.out_token) and torch.equal(so2.flags, so.flags)
+        assert torch.equal(so2.resid_mass, so.resid_mass)
+    ctx.close()
+
+
 def test_rows_above_m_are_never_read(cuda_device):
     """Rows m_b+1.. hold NaN: any touch would poison the sums."""
     w = _small("nan", B=32, gen_seed=0xBEEF70)
