@@ -457,15 +457,18 @@ __device__ __forceinline__ void decide_row(const VerifyArgs &a, int b, int r, in
     }
 }
 
-// The accepted prefix of sequence b from the rows' bits (one thread).
+// The accepted prefix of sequence b from the rows' bits, by warp 0: lane k holds
+// span_len[b, k] (loaded before the kernel waited), so nothing is loaded here.
 __device__ __forceinline__ void decide_prefix(const VerifyArgs &a, int b, int mb, bool bad_T,
-                                              const unsigned int *s_bits)
+                                              const unsigned int *s_bits, int lane, int32_t my_span)
 {
     const unsigned int all = s_bits[0];
     int n = 0;
     while (n < mb && (all >> n & 1u)) ++n;
-    int nd = 0;
-    for (int k = 0; k < n; ++k) nd += a.span_len[(size_t)b * a.K_max + k];
+    int nd = lane < n ? my_span : 0;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) nd += __shfl_xor_sync(0xFFFFFFFFu, nd, off);
+    if (lane != 0) return;
     uint32_t f = (all >> 16) & OD_VF_BOUNDARY_MASK;
     if (s_bits[1] & 1u) f |= OD_VF_NONFINITE;
     if (bad_T) { f |= OD_VF_BAD_TEMPERATURE; n = 0; nd = 0; }
@@ -518,6 +521,8 @@ od_verify_decide_kernel(const VerifyArgs a)
     const char *row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)r * a.row_stride) * ESZ;
     float x_t = 0.f, q = 0.f, u = 0.f;
     bool t_ok = false;
+    int32_t my_span = 0;                                     // warp 0, lane k: span_len[b, k]
+    if (!SHARD && r == 0 && lane < mb) my_span = a.span_len[(size_t)b * a.K_max + lane];
     if (lane == 0 && r < mb) {
         const size_t o = (size_t)b * a.K_max + r;
         const int32_t t = a.tgt_ids[o] - (SHARD ? a.col0 : 0);
@@ -560,7 +565,7 @@ od_verify_decide_kernel(const VerifyArgs a)
     }
     if (SHARD) return;
     __syncthreads();
-    if (threadIdx.x == 0) decide_prefix(a, b, mb, bad_T, s_bits);
+    if (r == 0) decide_prefix(a, b, mb, bad_T, s_bits, lane, my_span);
 }
 
 // Vocabulary shards, after the exchange: one block per sequence, warp r = row r merges
@@ -579,6 +584,8 @@ od_verify_finish_kernel(const VerifyArgs a)
     const float scale = bad_T ? 0.f : 1.4426950408889634f / T;
     float q = 0.f, u = 0.f;
     bool t_ok = false;
+    int32_t my_span = 0;
+    if (r == 0 && lane < mb) my_span = a.span_len[(size_t)b * a.K_max + lane];
     if (lane == 0 && r < mb) {
         const size_t o = (size_t)b * a.K_max + r;
         const int32_t t = a.tgt_ids[o];
@@ -604,7 +611,7 @@ od_verify_finish_kernel(const VerifyArgs a)
         if (lane == 0) decide_row(a, b, r, mb, c, s, mx, scale, t_ok, x_t, q, u, s_bits);
     }
     __syncthreads();
-    if (threadIdx.x == 0) decide_prefix(a, b, mb, bad_T, s_bits);
+    if (r == 0) decide_prefix(a, b, mb, bad_T, s_bits, lane, my_span);
 }
 
 template <typename Kern>
