@@ -472,12 +472,17 @@ od_sample_kernel(const SampleArgs a)
             if (t_hi > tile_hi) t_hi = tile_hi;
             if (t_lo < t_hi) warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val, dummy);
         }
-        __threadfence();                               // the tile values are read by another block
+        // The tile values are read by another block: the barrier orders this block's stores
+        // before thread 0's fence, the fence before its ticket (release); the block that
+        // draws the last ticket fences again before anyone in it reads (acquire).
         __syncthreads();
-        if (threadIdx.x == 0) s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
+        if (threadIdx.x == 0) {
+            __threadfence();
+            s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
+            __threadfence();
+        }
         __syncthreads();
         if (!s_last) return;
-        __threadfence();
     }
 
     // ---- pass 2 (one block per sequence) ----
