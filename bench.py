@@ -67,6 +67,7 @@ def parse():
     ap.add_argument("--verify-blocks-per-sm", type=int, default=0)
     ap.add_argument("--verify-waves", type=int, default=0)
     ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
+    ap.add_argument("--sample-dense", type=int, default=-1, help="sampler pass 1: 0 automatic, 1 lists, 2..4 inverse map with that many tiles in flight")
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches")
     return ap.parse_args()
 
@@ -469,6 +470,8 @@ def main():
         ctx.set_option("verify_waves", a.verify_waves)
     if a.sample_tiles_per_warp:
         ctx.set_option("sample_tiles_per_warp", a.sample_tiles_per_warp)
+    if a.sample_dense >= 0:
+        ctx.set_option("sample_dense", a.sample_dense)
     if a.no_pdl:
         ctx.set_option("pdl", 0)
 

@@ -270,6 +270,11 @@ int32_t od_set_option(od_ctx *c, const char *name, int64_t value)
     if (!strcmp(name, "verify_waves")) { c->opt_verify_waves = value; return OD_OK; }
     if (!strcmp(name, "sample_tiles_per_warp")) { c->opt_sample_tiles_per_warp = value; return OD_OK; }
     if (!strcmp(name, "pdl")) { c->opt_pdl = value != 0; return OD_OK; }
+    if (!strcmp(name, "sample_dense")) {
+        if (value > 4) return OD_ERR_INVALID_ARG;
+        c->opt_sample_dense = value;
+        return OD_OK;
+    }
     return OD_ERR_INVALID_ARG;
 }
 

@@ -75,6 +75,7 @@ struct SampleArgs {
     const double *mass_all;             // [n_shards][B][2] (residual share, share of p_j or 0)
     double *mass_out;                   // [B][2] this shard's shares
     int32_t early;                      // 1: the translation's outputs may be read before griddepcontrol.wait
+    int32_t dense;                      // pass 1 through the inverse map: tiles in flight per warp (0 = through the lists)
 };
 
 // what one sequence's warps need to evaluate r(t)
@@ -327,6 +328,38 @@ __device__ __forceinline__ void warp_tiles(const SeqState &q, const SampleArgs &
         warp_batch<DTYPE, TB>(q, a, residual, t, t_hi - t < TB ? t_hi - t : TB, lane, tile_val, dummy);
 }
 
+// Pass 1 without the lists: every id of a tile looks up its draft id in the inverse map
+// (coalesced) and gathers the drafter's probability if it has one. Per id this moves more
+// bytes than the lists do (the inverse map is twice the size of a bf16 row, but it stays in
+// L2), and it takes far fewer instructions per tile; NT tiles are in flight per warp.
+template <int DTYPE, int NT>
+__device__ __forceinline__ void warp_tiles_dense(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
+                                                 int t_hi, int lane, double *tile_val)
+{
+    for (int t = t_lo; t < t_hi; t += NT) {
+        float r[NT][EPT];
+#pragma unroll
+        for (int i = 0; i < NT; ++i) {
+            if (t + i < t_hi) {
+                if (residual) tile_values<DTYPE>(q, a, true, t + i, lane, r[i]);
+                else tile_e_values<DTYPE>(q, a, t + i, lane, r[i]);
+            }
+        }
+        float mine = 0.f;
+#pragma unroll
+        for (int i = 0; i < NT; ++i) {
+            if (t + i < t_hi) {
+                float s = r[i][0];
+#pragma unroll
+                for (int e = 1; e < EPT; ++e) s += r[i][e];
+                s = warp_sum_f32(s);
+                if (lane == i) mine = s;
+            }
+        }
+        if (lane < NT && t + lane < t_hi) tile_val[t + lane] = (double)mine;
+    }
+}
+
 // Sum of s_val[my_lo, my_hi) over the block's threads in the order of the scan of
 // pass 2 (a thread's run, lanes in order, warps in order); every thread gets it.
 __device__ __forceinline__ double block_total(const double *s_val, int my_lo, int my_hi, double *s_warp)
@@ -470,7 +503,12 @@ od_sample_kernel(const SampleArgs a)
             const int t_lo = tile_lo + (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
             int t_hi = t_lo + a.tiles_per_warp;
             if (t_hi > tile_hi) t_hi = tile_hi;
-            if (t_lo < t_hi) warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val, dummy);
+            if (t_lo < t_hi) {
+                if (a.dense == 2) warp_tiles_dense<DTYPE, 2>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
+                else if (a.dense == 3) warp_tiles_dense<DTYPE, 3>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
+                else if (a.dense == 4) warp_tiles_dense<DTYPE, 4>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
+                else warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val, dummy);
+            }
         }
         // The tile values are read by another block: the barrier orders this block's stores
         // before thread 0's fence, the fence before its ticket (release); the block that
@@ -705,6 +743,7 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     // the translation kernel releases its successor before it has written anything: directly
     // after it, nothing may be read early
     a.early = c->last_was_map ? 0 : 1;
+    a.dense = c->opt_sample_dense == 1 ? 0 : (c->opt_sample_dense >= 2 ? (int32_t)c->opt_sample_dense : 2);
     c->last_was_map = false;
     if (mode != 2) {
         c->info[2] = (int64_t)blocks_x * B;
