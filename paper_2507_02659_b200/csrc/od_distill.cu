@@ -61,7 +61,9 @@ __device__ __forceinline__ double block_sum(double v, double *s_red)
     return t;
 }
 
-template <int DTYPE>
+// VEC4: the draft vocabulary is a multiple of 4 and the rows are 16-byte aligned, so the
+// coalesced accesses (map, q, gradient) move four ids per instruction.
+template <int DTYPE, bool VEC4>
 __global__ void __launch_bounds__(THREADS, 2)
 od_distill_kernel(const DistillArgs a)
 {
@@ -118,35 +120,73 @@ od_distill_kernel(const DistillArgs a)
     // sum_d q(d) g(d). The loads of EB ids are issued together (map and q, then the
     // gathered logits). q(d) g(d) is parked in the gradient row itself (it stays in L2),
     // so that sweep 2 neither gathers nor takes a logarithm again.
-    constexpr int EB = 16;
     const bool park = grad != nullptr;
     float loss_t = 0.f, qg_t = 0.f;
-    for (int base = threadIdx.x; base < a.v_q; base += THREADS * EB) {
-        float qd[EB], x[EB];
-        {
-            int32_t t[EB];
+    // one id: q (negative = no map), its gathered logit -> the terms of the loss and of sum q g;
+    // returns q(d) g(d)
+    auto term = [&](float qs, float x) -> float {
+        const bool ok = qs >= FLT_MIN;                       // mapped and with (normal) mass
+        const float qa = fabsf(qs);
+        const float f = ok ? LN2 * (lg2_approx(qa) - fmaf(x - M, scale, -lg2_S)) : 0.f;
+        const float g = ok ? f + 1.f : 0.f;
+        loss_t += qa * f;
+        qg_t += qa * g;
+        return qa * g;
+    };
+    if (VEC4) {
+        constexpr int EV = 4;                                // vectors of 4 ids in flight per thread
+        for (int base = threadIdx.x * 4; base < a.v_q; base += THREADS * 4 * EV) {
+            int4 t[EV];
+            float4 qv[EV];
+#pragma unroll
+            for (int e = 0; e < EV; ++e) {
+                const int d = base + e * THREADS * 4;
+                t[e] = d < a.v_q ? __ldg((const int4 *)(a.vocab_map + d)) : make_int4(-1, -1, -1, -1);
+                qv[e] = d < a.v_q ? __ldg((const float4 *)(q + d)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            float x[EV][4];
+#pragma unroll
+            for (int e = 0; e < EV; ++e) {
+                x[e][0] = od_load_logit<DTYPE>(row, t[e].x >= 0 ? t[e].x : 0);
+                x[e][1] = od_load_logit<DTYPE>(row, t[e].y >= 0 ? t[e].y : 0);
+                x[e][2] = od_load_logit<DTYPE>(row, t[e].z >= 0 ? t[e].z : 0);
+                x[e][3] = od_load_logit<DTYPE>(row, t[e].w >= 0 ? t[e].w : 0);
+            }
+#pragma unroll
+            for (int e = 0; e < EV; ++e) {
+                const int d = base + e * THREADS * 4;
+                float4 o;
+                o.x = term(t[e].x < 0 ? -qv[e].x : qv[e].x, x[e][0]);
+                o.y = term(t[e].y < 0 ? -qv[e].y : qv[e].y, x[e][1]);
+                o.z = term(t[e].z < 0 ? -qv[e].z : qv[e].z, x[e][2]);
+                o.w = term(t[e].w < 0 ? -qv[e].w : qv[e].w, x[e][3]);
+                if (park && d < a.v_q) *(float4 *)(grad + d) = o;
+            }
+        }
+    } else {
+        constexpr int EB = 16;
+        for (int base = threadIdx.x; base < a.v_q; base += THREADS * EB) {
+            float qd[EB], x[EB];
+            {
+                int32_t t[EB];
+#pragma unroll
+                for (int e = 0; e < EB; ++e) {
+                    const int d = base + e * THREADS;
+                    t[e] = d < a.v_q ? __ldg(a.vocab_map + d) : -1;
+                    qd[e] = d < a.v_q ? __ldg(q + d) : 0.f;
+                }
+#pragma unroll
+                for (int e = 0; e < EB; ++e)                 // an id without a map: q = 0 drops its term below
+                    if (t[e] < 0) qd[e] = -qd[e];
+#pragma unroll
+                for (int e = 0; e < EB; ++e) x[e] = od_load_logit<DTYPE>(row, t[e] >= 0 ? t[e] : 0);
+            }
 #pragma unroll
             for (int e = 0; e < EB; ++e) {
                 const int d = base + e * THREADS;
-                t[e] = d < a.v_q ? __ldg(a.vocab_map + d) : -1;
-                qd[e] = d < a.v_q ? __ldg(q + d) : 0.f;
+                const float v = term(qd[e], x[e]);
+                if (park && d < a.v_q) grad[d] = v;
             }
-#pragma unroll
-            for (int e = 0; e < EB; ++e)                     // an id without a map: q = 0 drops its term below
-                if (t[e] < 0) qd[e] = -qd[e];
-#pragma unroll
-            for (int e = 0; e < EB; ++e) x[e] = od_load_logit<DTYPE>(row, t[e] >= 0 ? t[e] : 0);
-        }
-#pragma unroll
-        for (int e = 0; e < EB; ++e) {
-            const int d = base + e * THREADS;
-            const bool ok = qd[e] >= FLT_MIN;                // mapped and with (normal) mass
-            qd[e] = fabsf(qd[e]);
-            const float f = ok ? LN2 * (lg2_approx(qd[e]) - fmaf(x[e] - M, scale, -lg2_S)) : 0.f;
-            const float g = ok ? f + 1.f : 0.f;
-            loss_t += qd[e] * f;
-            qg_t += qd[e] * g;
-            if (park && d < a.v_q) grad[d] = qd[e] * g;
         }
     }
     const double loss = block_sum((double)loss_t, s_red);
@@ -156,8 +196,19 @@ od_distill_kernel(const DistillArgs a)
         // Sweep 2: grad(d) = q(d) g(d) - q(d) * sum_e q(e) g(e); every thread revisits the
         // ids it wrote itself, so no barrier is needed for the parked values
         const float gbar = (float)qg;
+        if (VEC4) {
 #pragma unroll 4
-        for (int d = threadIdx.x; d < a.v_q; d += THREADS) grad[d] = fmaf(-__ldg(q + d), gbar, grad[d]);
+            for (int d = threadIdx.x * 4; d < a.v_q; d += THREADS * 4) {
+                const float4 qq = __ldg((const float4 *)(q + d));
+                float4 gv = *(float4 *)(grad + d);
+                gv.x = fmaf(-qq.x, gbar, gv.x); gv.y = fmaf(-qq.y, gbar, gv.y);
+                gv.z = fmaf(-qq.z, gbar, gv.z); gv.w = fmaf(-qq.w, gbar, gv.w);
+                *(float4 *)(grad + d) = gv;
+            }
+        } else {
+#pragma unroll 4
+            for (int d = threadIdx.x; d < a.v_q; d += THREADS) grad[d] = fmaf(-__ldg(q + d), gbar, grad[d]);
+        }
     }
 }
 
@@ -178,7 +229,13 @@ cudaError_t od_launch_distill(od_ctx *c, int32_t B, int32_t K_max, const float *
     a.row_max = row_max; a.row_sum = row_sum; a.p_sel = p_sel; a.temperature = temperature;
     a.vocab_map = c->d_vocab_map; a.lambda = lambda; a.lambda_mode = lambda_mode; a.loss = loss; a.grad = grad;
     dim3 grid((unsigned)K_max, (unsigned)B);
-    if (dtype == OD_BF16) od_distill_kernel<OD_BF16><<<grid, THREADS, 0, s>>>(a);
-    else od_distill_kernel<OD_F32><<<grid, THREADS, 0, s>>>(a);
+    const bool vec4 = c->v_q % 4 == 0 && ((uintptr_t)q_rows & 15u) == 0 && (!grad || ((uintptr_t)grad & 15u) == 0);
+    if (dtype == OD_BF16) {
+        if (vec4) od_distill_kernel<OD_BF16, true><<<grid, THREADS, 0, s>>>(a);
+        else od_distill_kernel<OD_BF16, false><<<grid, THREADS, 0, s>>>(a);
+    } else {
+        if (vec4) od_distill_kernel<OD_F32, true><<<grid, THREADS, 0, s>>>(a);
+        else od_distill_kernel<OD_F32, false><<<grid, THREADS, 0, s>>>(a);
+    }
     return cudaGetLastError();
 }
