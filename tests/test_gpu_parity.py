@@ -101,6 +101,15 @@ def test_max_k_and_zero_length_proposals(cuda_device):
     assert s.sequences == 160
 
 
+def test_batches_beyond_one_verify_launch(cuda_device):
+    """od_verify handles at most 2048 sequences per launch and goes through longer batches in
+    slices: sequences on both sides of the cut are compared with the oracle."""
+    w = _small("slices", B=2500, v_q=300, v_p=777, cache_entries=100, gen_seed=0xBEEF55)
+    sel = np.concatenate([np.arange(0, 2500, 97), np.arange(2040, 2056), np.array([2499])])
+    s = _run_workload(w, cuda_device, [0], pad=True, sel=np.unique(sel))
+    assert s.sequences == len(np.unique(sel))
+
+
 # ------------------------------------------------------------ the five configs
 def test_config1_full_shape(cuda_device):
     w = synth.paper_config(1)
