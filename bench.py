@@ -159,6 +159,17 @@ def step_bytes(s):
     return sum(x.numel() * x.element_size() for x in t)
 
 
+def host_step_bytes(s, w):
+    """Bytes od_step_host copies to the device for step `s`: the small per-sequence arrays, and of
+    the logits and the drafter's distributions only the rows the step can read (rows 0..K_b and
+    0..K_b-1 of sequence b)."""
+    small = sum(x.numel() * x.element_size() for x in (s.draft_ids, s.draft_len, s.q_sel, s.temperature, s.seed))
+    kb = s.draft_len.clamp(0, w.k_max).long()
+    rows_l = int((kb + 1).sum())
+    rows_q = int(kb.sum())
+    return small + rows_l * w.v_p * s.logits.element_size() + rows_q * w.v_q * 4
+
+
 def oracle_time(w, st, host_steps, seconds):
     """Oracle on host cores over `host_steps` (CPU StepInputs, cycled), one full batch
     per step, until `seconds` have passed. Returns (tokens, elapsed_s, steps_done, threads)."""
@@ -612,7 +623,7 @@ def main():
                   (hout.n_accepted, hout.n_draft_accepted, hout.out_token, hout.tgt_ids, hout.m,
                    hout.verify_flags, hout.sample_flags))
         e2e = {"value": tok_e_all / (ms_e_max * 1e-3), "unit": UNIT, "steps": n_e,
-               "ms_per_step": ms_e_max / n_e, "h2d_bytes_per_step": step_bytes(hosts[0]),
+               "ms_per_step": ms_e_max / n_e, "h2d_bytes_per_step": host_step_bytes(hosts[0], w),
                "d2h_bytes_per_step": d2h, "api": "od_step_host (pinned host buffers)"}
 
     cpu = None

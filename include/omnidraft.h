@@ -371,7 +371,9 @@ int32_t od_host_step_reserve(od_ctx *ctx, int32_t logit_dtype);
 /* Steps 1-3 on HOST buffers (pinned memory recommended): copies the inputs to
  * the staging area, runs the three kernels, copies the results back, all on
  * `stream`, and synchronises that stream before returning. Host layouts are
- * the dense ones above (logits [B, K_max+1, target_vocab]). Outputs: host
+ * the dense ones above (logits [B, K_max+1, target_vocab]); of the logits and
+ * of q_rows only the rows the step can read are copied (rows 0..K_b and
+ * 0..K_b-1 of sequence b, K_b = draft_len[b] read on the host). Outputs: host
  * int32[B] each for n_accepted, n_draft_accepted, out_token; int32[B,K_max]
  * tgt_ids; int32[B] m; uint32[B] verify_flags and sample_flags (any output may
  * be NULL). Needs od_host_step_reserve with the same dtype. */

@@ -551,8 +551,30 @@ int32_t od_step_host(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_i
     OD_CUDA(cudaMemcpyAsync(c->s_q_sel, q_sel, nB * K * 4, H2D, s));
     OD_CUDA(cudaMemcpyAsync(c->s_temperature, temperature, nB * 4, H2D, s));
     OD_CUDA(cudaMemcpyAsync(c->s_seed, seed, nB * 8, H2D, s));
-    OD_CUDA(cudaMemcpyAsync(c->s_logits, logits, nB * (K + 1) * (size_t)c->v_p * esz, H2D, s));
-    OD_CUDA(cudaMemcpyAsync(c->s_q_rows, q_rows, nB * K * (size_t)c->v_q * 4, H2D, s));
+    // Only the rows the step can read cross the bus: logit rows 0..K_b and drafter rows
+    // 0..K_b-1 of sequence b (m_b <= K_b). Neighbouring sequences with full proposals
+    // merge into one copy; the rest of the staging buffers keeps earlier contents, which
+    // no kernel looks at.
+    {
+        const size_t lrow = (size_t)c->v_p * esz, qrow = (size_t)c->v_q * 4;
+        size_t l_from = 0, l_bytes = 0, q_from = 0, q_bytes = 0;   // pending runs (byte offsets)
+        for (size_t b = 0; b <= nB; ++b) {
+            int32_t kb = 0;
+            if (b < nB) { kb = draft_len[b]; kb = kb < 0 ? 0 : (kb > K_max ? K_max : kb); }
+            const size_t l_at = b * (K + 1) * lrow, q_at = b * K * qrow;
+            if (b == nB || l_from + l_bytes != l_at) {
+                if (l_bytes)
+                    OD_CUDA(cudaMemcpyAsync((char *)c->s_logits + l_from, (const char *)logits + l_from, l_bytes, H2D, s));
+                l_from = l_at; l_bytes = 0;
+            }
+            if (b == nB || q_from + q_bytes != q_at) {
+                if (q_bytes)
+                    OD_CUDA(cudaMemcpyAsync((char *)c->s_q_rows + q_from, (const char *)q_rows + q_from, q_bytes, H2D, s));
+                q_from = q_at; q_bytes = 0;
+            }
+            if (b < nB) { l_bytes += (size_t)(kb + 1) * lrow; q_bytes += (size_t)kb * qrow; }
+        }
+    }
     OD_CUDA(od_launch_map(c, B, K_max, c->s_draft_ids, c->s_draft_len, c->s_q_sel, c->s_tgt_ids,
                           c->s_q_prime, c->s_span_start, c->s_span_len, c->s_m, c->s_tail, nullptr, s));
     OD_CUDA(od_launch_verify(c, B, K_max, c->s_logits, logit_dtype, row_stride, seq_stride,
