@@ -67,7 +67,7 @@ def parse():
     ap.add_argument("--verify-blocks-per-sm", type=int, default=0)
     ap.add_argument("--verify-waves", type=int, default=0)
     ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
-    ap.add_argument("--sample-dense", type=int, default=-1, help="sampler pass 1: 0 automatic, 1 lists, 2..4 inverse map with that many tiles in flight")
+    ap.add_argument("--sample-dense", type=int, default=-1, help="sampler pass 1: 0 automatic, 1 lists, 2..4 inverse map with that many tiles in flight, 5 pipelined pairs")
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches")
     return ap.parse_args()
 

@@ -185,7 +185,8 @@ int32_t od_cache_dump(od_ctx *ctx, int64_t max_out, int32_t *runs, int32_t *len,
  * 0 = automatic), "sample_dense" (how the first pass of od_sample_residual finds
  * the drafter's probability of a target id: 1 = through per-tile lists of the mapped
  * ids, 2..4 = through the inverse map with that many tiles in flight per warp,
- * 0 = automatic), "pdl" (1 = launch the step kernels with programmatic stream
+ * 5 = through the inverse map, pairs of tiles software-pipelined, 0 = automatic),
+ * "pdl" (1 = launch the step kernels with programmatic stream
  * serialization so that a kernel's prologue overlaps its predecessor's tail,
  * the default; 0 = plain stream order). Unknown name: INVALID_ARG. */
 int32_t od_set_option(od_ctx *ctx, const char *name, int64_t value);

@@ -271,7 +271,7 @@ int32_t od_set_option(od_ctx *c, const char *name, int64_t value)
     if (!strcmp(name, "sample_tiles_per_warp")) { c->opt_sample_tiles_per_warp = value; return OD_OK; }
     if (!strcmp(name, "pdl")) { c->opt_pdl = value != 0; return OD_OK; }
     if (!strcmp(name, "sample_dense")) {
-        if (value > 4) return OD_ERR_INVALID_ARG;
+        if (value > 5) return OD_ERR_INVALID_ARG;
         c->opt_sample_dense = value;
         return OD_OK;
     }

@@ -62,7 +62,7 @@ struct od_ctx {
     int64_t opt_verify_blocks_per_sm;
     int64_t opt_verify_waves;       // grid = waves x the resident capacity (experiments)
     int64_t opt_sample_tiles_per_warp;
-    int64_t opt_sample_dense;       // pass 1 of the sampler: 0 = automatic, 1 = lists, 2..4 = inverse map, that many tiles in flight
+    int64_t opt_sample_dense;       // pass 1 of the sampler: 0 = automatic, 1 = lists, 2..4 = inverse map, that many tiles in flight, 5 = pipelined pairs
     int64_t opt_pdl;                // launch with programmatic stream serialization
 
     // the last launch on this context was the translation kernel, which lets the next

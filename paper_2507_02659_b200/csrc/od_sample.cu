@@ -75,7 +75,7 @@ struct SampleArgs {
     const double *mass_all;             // [n_shards][B][2] (residual share, share of p_j or 0)
     double *mass_out;                   // [B][2] this shard's shares
     int32_t early;                      // 1: the translation's outputs may be read before griddepcontrol.wait
-    int32_t dense;                      // pass 1 through the inverse map: tiles in flight per warp (0 = through the lists)
+    int32_t dense;                      // pass 1: 0 = through the lists, 2..4 = inverse map, that many tiles in flight, 5 = pipelined pairs
 };
 
 // what one sequence's warps need to evaluate r(t)
@@ -98,6 +98,25 @@ struct SeqState {
 __device__ __forceinline__ float resid_of(const SeqState &q, float x, float qq)
 {
     return fmaxf(0.f, fmaf(-qq, q.S, od_ex2(fmaf(x, q.scale, -q.c))));
+}
+
+// Eq. (2): the two ids whose q' is not the drafter's row. Only the lane that owns such
+// an id (its ids are t0 .. t0 + EPT - 1) redoes it: prefix sub-token first, the n-gram
+// token last.
+template <int DTYPE>
+__device__ __forceinline__ void eq2_ids(const SeqState &q, const SampleArgs &a, int t0, float *r)
+{
+    const int dp = q.prefix_token - t0, dn = q.ngram_token - t0;
+    if ((unsigned)dp < (unsigned)EPT && q.prefix_token < a.v_p) {
+        const float v = resid_of(q, od_load_logit<DTYPE>(q.row, q.prefix_token), q.prefix_val);
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) r[e] = e == dp ? v : r[e];
+    }
+    if ((unsigned)dn < (unsigned)EPT && q.ngram_token < a.v_p) {
+        const float v = resid_of(q, od_load_logit<DTYPE>(q.row, q.ngram_token), q.ngram_prob);
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) r[e] = e == dn ? v : r[e];
+    }
 }
 
 // r'(t) of the EPT consecutive ids this lane owns in `tile`; ids >= v_p give 0
@@ -147,21 +166,7 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
             }
         }
     }
-    if (residual) {
-        // Eq. (2): the two ids whose q' is not the drafter's row. Only the lane that
-        // owns such an id redoes it (prefix sub-token first, the n-gram token last).
-        const int dp = q.prefix_token - t0, dn = q.ngram_token - t0;
-        if ((unsigned)dp < (unsigned)EPT && q.prefix_token < a.v_p) {
-            const float v = resid_of(q, od_load_logit<DTYPE>(q.row, q.prefix_token), q.prefix_val);
-#pragma unroll
-            for (int e = 0; e < EPT; ++e) r[e] = e == dp ? v : r[e];
-        }
-        if ((unsigned)dn < (unsigned)EPT && q.ngram_token < a.v_p) {
-            const float v = resid_of(q, od_load_logit<DTYPE>(q.row, q.ngram_token), q.ngram_prob);
-#pragma unroll
-            for (int e = 0; e < EPT; ++e) r[e] = e == dn ? v : r[e];
-        }
-    }
+    if (residual) eq2_ids<DTYPE>(q, a, t0, r);
 }
 
 // a lane's eight values are added in fp32 in index order (both passes do exactly
@@ -360,6 +365,76 @@ __device__ __forceinline__ void warp_tiles_dense(const SeqState &q, const Sample
     }
 }
 
+// The same pass for a residual draw, software-pipelined over pairs of WHOLE tiles: the
+// inverse-map entries of the next pair are requested before the current pair's gathers,
+// so a pair costs one memory round trip, not two.
+template <int DTYPE>
+__device__ __forceinline__ void warp_tiles_dense_piped(const SeqState &q, const SampleArgs &a, int t_lo, int t_hi,
+                                                       int lane, double *tile_val)
+{
+    constexpr int ESZ = DTYPE == OD_BF16 ? 2 : 4;
+    int4 ni[2][2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int t0 = (t_lo + i < t_hi ? t_lo + i : t_lo) * OD_SAMPLE_TILE + lane * EPT;
+        ni[i][0] = __ldg((const int4 *)(a.inv_map + t0));
+        ni[i][1] = __ldg((const int4 *)(a.inv_map + t0) + 1);
+    }
+    for (int t = t_lo; t < t_hi; t += 2) {
+        int32_t d[2][EPT];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            d[i][0] = ni[i][0].x; d[i][1] = ni[i][0].y; d[i][2] = ni[i][0].z; d[i][3] = ni[i][0].w;
+            d[i][4] = ni[i][1].x; d[i][5] = ni[i][1].y; d[i][6] = ni[i][1].z; d[i][7] = ni[i][1].w;
+        }
+        if (t + 2 < t_hi) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int t0 = (t + 2 + i < t_hi ? t + 2 + i : t + 2) * OD_SAMPLE_TILE + lane * EPT;
+                ni[i][0] = __ldg((const int4 *)(a.inv_map + t0));
+                ni[i][1] = __ldg((const int4 *)(a.inv_map + t0) + 1);
+            }
+        }
+        const bool two = t + 1 < t_hi;
+        uint4 raw[2][DTYPE == OD_BF16 ? 1 : 2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint4 *src = (const uint4 *)(q.row + (size_t)((i == 0 || two ? t + i : t) * OD_SAMPLE_TILE + lane * EPT) * ESZ);
+            raw[i][0] = __ldg(src);
+            if (DTYPE != OD_BF16) raw[i][1] = __ldg(src + 1);
+        }
+        float qq[2][EPT];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) qq[i][e] = d[i][e] >= 0 ? __ldg(q.q_row + d[i][e]) : 0.f;
+        }
+        float mine = 0.f;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            float x[EPT], r[EPT];
+            if (DTYPE == OD_BF16) {
+                const uint4 v = raw[i][0];
+                x[0] = od_bf16_lo(v.x); x[1] = od_bf16_hi(v.x); x[2] = od_bf16_lo(v.y); x[3] = od_bf16_hi(v.y);
+                x[4] = od_bf16_lo(v.z); x[5] = od_bf16_hi(v.z); x[6] = od_bf16_lo(v.w); x[7] = od_bf16_hi(v.w);
+            } else {
+                const uint4 v0 = raw[i][0], v1 = raw[i][DTYPE == OD_BF16 ? 0 : 1];
+                x[0] = __uint_as_float(v0.x); x[1] = __uint_as_float(v0.y); x[2] = __uint_as_float(v0.z); x[3] = __uint_as_float(v0.w);
+                x[4] = __uint_as_float(v1.x); x[5] = __uint_as_float(v1.y); x[6] = __uint_as_float(v1.z); x[7] = __uint_as_float(v1.w);
+            }
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) r[e] = resid_of(q, x[e], qq[i][e]);
+            eq2_ids<DTYPE>(q, a, (t + i) * OD_SAMPLE_TILE + lane * EPT, r);
+            float sum = r[0];
+#pragma unroll
+            for (int e = 1; e < EPT; ++e) sum += r[e];
+            sum = warp_sum_f32(sum);
+            if (lane == i) mine = sum;
+        }
+        if (lane < 2 && t + lane < t_hi) tile_val[t + lane] = (double)mine;
+    }
+}
+
 // Sum of s_val[my_lo, my_hi) over the block's threads in the order of the scan of
 // pass 2 (a thread's run, lanes in order, warps in order); every thread gets it.
 __device__ __forceinline__ double block_total(const double *s_val, int my_lo, int my_hi, double *s_warp)
@@ -504,7 +579,17 @@ od_sample_kernel(const SampleArgs a)
             int t_hi = t_lo + a.tiles_per_warp;
             if (t_hi > tile_hi) t_hi = tile_hi;
             if (t_lo < t_hi) {
-                if (a.dense == 2) warp_tiles_dense<DTYPE, 2>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
+                if (a.dense == 5) {
+                    // whole tiles pipelined; the row's ragged last tile (if it is this warp's) on its own
+                    const int whole = a.v_p / OD_SAMPLE_TILE;
+                    const int hi_w = t_hi < whole ? t_hi : whole;
+                    if (q.residual) {
+                        if (t_lo < hi_w) warp_tiles_dense_piped<DTYPE>(q, a, t_lo, hi_w, lane, tile_val);
+                        if (hi_w < t_hi) warp_tiles_dense<DTYPE, 2>(q, a, true, hi_w > t_lo ? hi_w : t_lo, t_hi, lane, tile_val);
+                    } else {
+                        warp_tiles_dense<DTYPE, 2>(q, a, false, t_lo, t_hi, lane, tile_val);
+                    }
+                } else if (a.dense == 2) warp_tiles_dense<DTYPE, 2>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
                 else if (a.dense == 3) warp_tiles_dense<DTYPE, 3>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
                 else if (a.dense == 4) warp_tiles_dense<DTYPE, 4>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
                 else warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val, dummy);
@@ -743,7 +828,7 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     // the translation kernel releases its successor before it has written anything: directly
     // after it, nothing may be read early
     a.early = c->last_was_map ? 0 : 1;
-    a.dense = c->opt_sample_dense == 1 ? 0 : (c->opt_sample_dense >= 2 ? (int32_t)c->opt_sample_dense : 2);
+    a.dense = c->opt_sample_dense == 1 ? 0 : (c->opt_sample_dense >= 2 ? (int32_t)c->opt_sample_dense : 5);
     c->last_was_map = false;
     if (mode != 2) {
         c->info[2] = (int64_t)blocks_x * B;

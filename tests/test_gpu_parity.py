@@ -79,7 +79,7 @@ def test_cache_hits_and_unmapped_stops_are_exercised(cuda_device):
 
 
 @pytest.mark.parametrize("blocks_per_sm,tiles,pdl,dense", [(1, 1, 1, 1), (2, 2, 0, 2), (4, 7, 1, 3), (8, 1000, 0, 4),
-                                                           (4, 5, 1, 0)])
+                                                           (4, 5, 1, 0), (4, 3, 1, 5)])
 def test_every_split_of_a_row_gives_the_same_answer(cuda_device, blocks_per_sm, tiles, pdl, dense):
     w = _small("split", v_q=3000, v_p=20011, B=5, cache_entries=500, gen_seed=0xBEEF40)
     _run_workload(w, cuda_device, range(3), pad=True,
@@ -87,7 +87,7 @@ def test_every_split_of_a_row_gives_the_same_answer(cuda_device, blocks_per_sm, 
                         "sample_dense": dense})
 
 
-@pytest.mark.parametrize("dense", [1, 2])
+@pytest.mark.parametrize("dense", [1, 2, 5])
 def test_both_first_passes_of_the_sampler_on_the_batched_shape(cuda_device, dense):
     """The sampler's tile sums through the lists of mapped ids and through the inverse map."""
     w = synth.scaled(synth.paper_config(4), B=48, gen_seed=0xBEEF49)
