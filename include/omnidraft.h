@@ -29,7 +29,18 @@
  *     words, never by a trap.
  *   - A context holds scratch that its kernels share: calls on one context
  *     must be ordered (one stream, or explicit dependencies). Use one context
- *     per concurrent stream.
+ *     per concurrent stream, and make the calls of one step on one context.
+ *   - With option "pdl" = 1 (the default) the step kernels are launched with
+ *     programmatic stream serialization and start work on their INPUTS before
+ *     the launch in front of them in the stream has finished: od_verify reads
+ *     logits and temperatures early, od_sample_residual the outputs of
+ *     od_map_proposals (not when the call in front of it on its context was
+ *     od_map_proposals itself). So the step's inputs (draft ids, lengths and
+ *     probabilities, logits, temperatures, seeds) must be complete before the
+ *     launch that precedes the step's first call is enqueued; a producer that
+ *     is itself the preceding launch is fine if it is an ordinary kernel launch
+ *     (it has finished by the time a dependent kernel starts). "pdl" = 0 gives
+ *     plain stream order.
  *   - Positions: arrays indexed [B, K_max] hold K_max entries per sequence,
  *     of which the first K_b (inputs) or m_b (outputs) are meaningful.
  *   - Random numbers: Philox4x32-10 (Salmon et al., SC'11) with key = the
