@@ -88,9 +88,16 @@ def emulate_step(ctx: od.Context, logits: torch.Tensor, n_shards: int, mp: od.Ma
     v_p = logits.shape[2]
     bounds = [split_vocab(v_p, r, n_shards) for r in range(n_shards)]
     parts: List[torch.Tensor] = []
+    per16 = 16 // logits.element_size()
     for lo, hi in bounds:
         v = logits[:, :, lo:hi]
-        parts.append(v.contiguous() if copy_shards else v)
+        if copy_shards:
+            # a buffer of its own whose rows start on 16-byte boundaries (the last shard's length is arbitrary)
+            width = (hi - lo + per16 - 1) // per16 * per16
+            buf = torch.zeros(v.shape[0], v.shape[1], width, dtype=v.dtype, device=v.device)
+            buf[:, :, :hi - lo] = v
+            v = buf[:, :, :hi - lo]
+        parts.append(v)
     stats_all = torch.stack([od.od_verify_shard_stats(ctx, lo, p, mp, temperature)
                              for (lo, _), p in zip(bounds, parts)])
     vo = od.od_verify_shard_finish(ctx, stats_all, mp, temperature, seed, step_index)
