@@ -71,3 +71,19 @@ def test_full_vocabulary_sampled_sequences(cuda_device):
     """The batched 128256-id shape; the oracle recomputes a few sequences."""
     w = synth.scaled(synth.paper_config(4), B=16, name="cfg4-distill")
     _check(w, cuda_device, [0], 0.2, ds.LAMBDA_CONSTANT, positions=[0, 5, 11])
+
+
+@pytest.mark.parametrize("i", range(8))
+def test_random_shapes(cuda_device, i):
+    """Seeded random vocabulary sizes (both the 128-bit path, V_q a multiple of 4, and the scalar one),
+    proposal lengths, maps and temperatures."""
+    rng = np.random.default_rng(7000 + i)
+    v_q = int(rng.integers(50, 2500))
+    if i % 2 == 0:
+        v_q = v_q // 4 * 4
+    v_p = int(rng.integers(v_q, 5000))
+    k_max = int(rng.integers(1, 9))
+    w = _small(B=int(rng.integers(1, 12)), k_max=k_max, k_min=int(rng.integers(1, k_max + 1)), v_q=v_q, v_p=v_p,
+               logit_dtype=["bf16", "f32"][int(rng.integers(0, 2))], mapped_frac=float(rng.uniform(0.3, 0.9)),
+               cache_entries=int(rng.integers(0, 200)), gen_seed=0xBEEFE0 + i)
+    _check(w, cuda_device, range(2), lam=float(rng.uniform(0.05, 1.0)), mode=int(rng.integers(0, 2)))
