@@ -15,9 +15,9 @@
 //           come first in the order (inserted at the current clock?, score, run key)
 //           are dropped, score = last-access clock (LRU) or frequency (LFU). The
 //           k-th smallest is found by a most-significant-digit radix select over the
-//           104-bit order key (13 passes of a histogram kernel and a one-block
-//           select kernel, no sorting); then the survivors are re-inserted into the
-//           spare table, which becomes the table. No kernel waits for another.
+//           104-bit order key (13 passes of a histogram kernel whose last block to
+//           finish picks the digit, no sorting); then the survivors are re-inserted
+//           into the spare table, which becomes the table. No kernel waits for another.
 #include <string.h>
 #include <utility>
 #include <vector>
@@ -34,6 +34,7 @@ struct TrimState {
     unsigned long long pre_hi, pre_lo, mask_hi, mask_lo;   // decided digits of the k-th order key
     unsigned int hist[256];
     unsigned int invalid;       // malformed candidates seen by od_cache_insert
+    unsigned int ticket;        // blocks of the running histogram pass that are done
 };
 
 constexpr int PASSES = 13;      // 5 bytes of (new?, score), 8 bytes of the run key
@@ -112,6 +113,7 @@ __global__ void trim_begin_kernel(TrimState *st, unsigned int max_entries)
     st->k_rem = st->k;
     st->pre_hi = st->pre_lo = st->mask_hi = st->mask_lo = 0ull;
     for (int i = 0; i < 256; ++i) st->hist[i] = 0u;
+    st->ticket = 0u;
 }
 
 __global__ void trim_hist_kernel(int pass, int policy, unsigned int clock, const unsigned long long *keys,
@@ -123,47 +125,87 @@ __global__ void trim_hist_kernel(int pass, int policy, unsigned int clock, const
     s_hist[threadIdx.x] = 0u;
     __syncthreads();
     const unsigned long long pre_hi = st->pre_hi, pre_lo = st->pre_lo, m_hi = st->mask_hi, m_lo = st->mask_lo;
-    for (int64_t slot = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; slot < cap;
-         slot += (int64_t)gridDim.x * blockDim.x) {
-        const unsigned long long key = keys[slot];
-        if (key == 0ull || vals[slot] < 0) continue;
-        unsigned long long hi, lo;
-        order_key(policy, clock, key, stamp[slot], freq[slot], born[slot], hi, lo);
-        if ((hi & m_hi) == pre_hi && (lo & m_lo) == pre_lo) {
-            // scores are heavily tied (most digits are equal across the table): one
-            // shared-memory add per distinct digit of the warp, not one per entry
-            const unsigned int d = digit_of(pass, hi, lo);
-            const unsigned int peers = __match_any_sync(__activemask(), d);
-            if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&s_hist[d], (unsigned int)__popc(peers));
+    // four consecutive slots per thread and iteration, every load issued before the first
+    // use: the pass is a chain of memory round trips otherwise (the table sits in L2)
+    const unsigned int *score = policy == 0 ? stamp : freq;
+    for (int64_t slot = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; slot < cap;
+         slot += (int64_t)gridDim.x * blockDim.x * 4) {
+        const ulonglong2 k01 = __ldg((const ulonglong2 *)(keys + slot));
+        const ulonglong2 k23 = __ldg((const ulonglong2 *)(keys + slot) + 1);
+        const int4 v4 = __ldg((const int4 *)(vals + slot));
+        const uint4 s4 = __ldg((const uint4 *)(score + slot));
+        const uint4 b4 = __ldg((const uint4 *)(born + slot));
+        const unsigned long long kk[4] = {k01.x, k01.y, k23.x, k23.y};
+        const int vv[4] = {v4.x, v4.y, v4.z, v4.w};
+        const unsigned int ss[4] = {s4.x, s4.y, s4.z, s4.w};
+        const unsigned int bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (kk[e] == 0ull || vv[e] < 0) continue;
+            const unsigned long long hi = ((unsigned long long)(bb[e] == clock ? 1u : 0u) << 32) | ss[e], lo = kk[e];
+            if ((hi & m_hi) == pre_hi && (lo & m_lo) == pre_lo) {
+                // scores are heavily tied (most digits are equal across the table): one
+                // shared-memory add per distinct digit of the warp, not one per entry
+                const unsigned int d = digit_of(pass, hi, lo);
+                const unsigned int peers = __match_any_sync(__activemask(), d);
+                if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&s_hist[d], (unsigned int)__popc(peers));
+            }
         }
     }
     __syncthreads();
     if (s_hist[threadIdx.x]) atomicAdd(&st->hist[threadIdx.x], s_hist[threadIdx.x]);
-}
 
-// one block of 256 threads: the digit in which the running count reaches k_rem
-__global__ void trim_select_kernel(int pass, TrimState *st)
-{
-    __shared__ unsigned int s_cum[256];
-    if (st->k == 0u) return;
-    s_cum[threadIdx.x] = st->hist[threadIdx.x];
+    // The block that finishes last picks the digit in which the running count reaches
+    // k_rem (no second launch per pass): the barrier orders this block's adds before
+    // thread 0's fence and ticket; the last block fences again before it reads.
+    __shared__ unsigned int s_last;
     __syncthreads();
     if (threadIdx.x == 0) {
-        unsigned int run = 0, k_rem = st->k_rem, d = 255;
-        for (int i = 0; i < 256; ++i) {
-            if (run + s_cum[i] >= k_rem) { d = i; break; }
-            run += s_cum[i];
-        }
-        st->k_rem = k_rem - run;
-        if (pass < 5) {
-            st->pre_hi |= (unsigned long long)d << (8 * (4 - pass));
-            st->mask_hi |= 0xFFull << (8 * (4 - pass));
-        } else {
-            st->pre_lo |= (unsigned long long)d << (8 * (12 - pass));
-            st->mask_lo |= 0xFFull << (8 * (12 - pass));
-        }
+        __threadfence();
+        s_last = atomicAdd(&st->ticket, 1u) == gridDim.x - 1 ? 1u : 0u;
+        __threadfence();
     }
     __syncthreads();
+    if (!s_last) return;
+    s_hist[threadIdx.x] = __ldcg(&st->hist[threadIdx.x]);
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        // warp 0: lane l owns bins 8l .. 8l+7; the first bin at which the running count reaches k_rem
+        const int lane = threadIdx.x;
+        const unsigned int k_rem = st->k_rem;
+        unsigned int mine = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mine += s_hist[lane * 8 + i];
+        unsigned int inc = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned int t = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+            if (lane >= off) inc += t;
+        }
+        const unsigned int reach = __ballot_sync(0xFFFFFFFFu, inc >= k_rem);
+        const int owner = reach ? __ffs(reach) - 1 : 31;
+        unsigned int run = inc - mine, d = 255;
+        if (lane == owner) {
+            for (int i = 0; i < 8; ++i) {
+                if (run + s_hist[lane * 8 + i] >= k_rem) { d = lane * 8 + i; break; }
+                run += s_hist[lane * 8 + i];
+            }
+            if (d == 255u && !reach) run = inc;             // counts fell short: everything below the last bin
+        }
+        d = __shfl_sync(0xFFFFFFFFu, d, owner);
+        run = __shfl_sync(0xFFFFFFFFu, run, owner);
+        if (lane == 0) {
+            st->k_rem = k_rem - run;
+            if (pass < 5) {
+                st->pre_hi |= (unsigned long long)d << (8 * (4 - pass));
+                st->mask_hi |= 0xFFull << (8 * (4 - pass));
+            } else {
+                st->pre_lo |= (unsigned long long)d << (8 * (12 - pass));
+                st->mask_lo |= 0xFFull << (8 * (12 - pass));
+            }
+            st->ticket = 0u;
+        }
+    }
     st->hist[threadIdx.x] = 0u;
 }
 
@@ -187,27 +229,42 @@ __global__ void trim_rebuild_kernel(int policy, unsigned int clock, const unsign
     const unsigned int k = st->k;
     const unsigned long long thr_hi = st->pre_hi, thr_lo = st->pre_lo;
     const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
-    for (int64_t slot = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; slot < cap;
-         slot += (int64_t)gridDim.x * blockDim.x) {
-        const unsigned long long key = keys[slot];
-        if (key == 0ull || vals[slot] < 0) continue;
-        if (k > 0u) {
-            unsigned long long hi, lo;
-            order_key(policy, clock, key, stamp[slot], freq[slot], born[slot], hi, lo);
-            if (hi < thr_hi || (hi == thr_hi && lo <= thr_lo)) continue;   // among the k first: dropped
-        }
-        uint64_t g = od_hash64(key) & (ngroups - 1);
-        bool placed = false;
-        for (uint64_t step = 0; step < ngroups && !placed; ++step) {
-            for (int s = 0; s < OD_GROUP; ++s) {
-                const int64_t ns = (int64_t)(g * OD_GROUP + s);
-                if (nkeys[ns] == 0ull && atomicCAS(nkeys + ns, 0ull, key) == 0ull) {
-                    nvals[ns] = vals[slot]; nstamp[ns] = stamp[slot]; nfreq[ns] = freq[slot]; nborn[ns] = born[slot];
-                    placed = true;
-                    break;
-                }
+    for (int64_t slot4 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; slot4 < cap;
+         slot4 += (int64_t)gridDim.x * blockDim.x * 4) {
+        // as in the histogram pass: four slots, all loads first
+        const ulonglong2 k01 = __ldg((const ulonglong2 *)(keys + slot4));
+        const ulonglong2 k23 = __ldg((const ulonglong2 *)(keys + slot4) + 1);
+        const int4 v4 = __ldg((const int4 *)(vals + slot4));
+        const uint4 s4 = __ldg((const uint4 *)(stamp + slot4));
+        const uint4 f4 = __ldg((const uint4 *)(freq + slot4));
+        const uint4 b4 = __ldg((const uint4 *)(born + slot4));
+        const unsigned long long kk[4] = {k01.x, k01.y, k23.x, k23.y};
+        const int vv[4] = {v4.x, v4.y, v4.z, v4.w};
+        const unsigned int ss[4] = {s4.x, s4.y, s4.z, s4.w};
+        const unsigned int ff[4] = {f4.x, f4.y, f4.z, f4.w};
+        const unsigned int bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const unsigned long long key = kk[e];
+            if (key == 0ull || vv[e] < 0) continue;
+            if (k > 0u) {
+                unsigned long long hi, lo;
+                order_key(policy, clock, key, ss[e], ff[e], bb[e], hi, lo);
+                if (hi < thr_hi || (hi == thr_hi && lo <= thr_lo)) continue;   // among the k first: dropped
             }
-            g = (g + 1) & (ngroups - 1);
+            uint64_t g = od_hash64(key) & (ngroups - 1);
+            bool placed = false;
+            for (uint64_t step = 0; step < ngroups && !placed; ++step) {
+                for (int sl = 0; sl < OD_GROUP; ++sl) {
+                    const int64_t ns = (int64_t)(g * OD_GROUP + sl);
+                    if (nkeys[ns] == 0ull && atomicCAS(nkeys + ns, 0ull, key) == 0ull) {
+                        nvals[ns] = vv[e]; nstamp[ns] = ss[e]; nfreq[ns] = ff[e]; nborn[ns] = bb[e];
+                        placed = true;
+                        break;
+                    }
+                }
+                g = (g + 1) & (ngroups - 1);
+            }
         }
     }
 }
@@ -336,7 +393,6 @@ int32_t od_cache_trim(od_ctx *c, void *stream)
     for (int pass = 0; pass < PASSES; ++pass) {
         trim_hist_kernel<<<grid, 256, 0, s>>>(pass, c->dyn_policy, c->clock, (const unsigned long long *)c->d_keys,
                                               c->d_vals, c->d_stamp, c->d_freq, c->d_born, c->cap, st);
-        trim_select_kernel<<<1, 256, 0, s>>>(pass, st);
     }
     table_clear_kernel<<<grid, 256, 0, s>>>((unsigned long long *)c->d_keys2, c->d_vals2, c->d_stamp2,
                                             c->d_freq2, c->d_born2, c->cap);
