@@ -45,6 +45,11 @@ class Workload:
     gen_seed: int               # seed of the generator stream
     unmapped_shift: float = 4.0  # draft-logit penalty on ids with no direct map
     sigma: float = 3.0
+    # Cache targets normally lie outside the map's image (a token whose text is one draft
+    # token does not come back as a run). These shares put some inside it, to exercise the
+    # collisions between the cases of Eq. (2):
+    targets_in_image: float = 0.0    # share of entries whose target has a direct pre-image
+    targets_on_prefix: float = 0.0   # share whose target is the image of the run's first id
 
 
 def paper_config(i: int) -> Workload:
@@ -157,7 +162,9 @@ def make_static(w: Workload) -> Static:
         in_image[vocab_map[vocab_map >= 0]] = True
         outside = np.nonzero(~in_image)[0]
         if outside.size == 0:
-            raise ValueError("cache targets need target ids outside the map's image")
+            if w.targets_in_image + w.targets_on_prefix < 1.0:
+                raise ValueError("cache targets need target ids outside the map's image")
+            outside = np.arange(w.v_p)
         # distinct runs: draw, pack, de-duplicate, top up
         have = 0
         seen = set()
@@ -179,6 +186,15 @@ def make_static(w: Workload) -> Static:
         # several runs may share a target token: the cache can hold more
         # entries than there are target ids outside the image
         run_target[:] = outside[rng.integers(0, outside.size, size=E)]
+        if w.targets_in_image > 0 or w.targets_on_prefix > 0:
+            image = np.nonzero(in_image)[0]
+            coin = rng.random(E)
+            pick = image[rng.integers(0, max(1, image.size), size=E)] if image.size else run_target
+            first = vocab_map[runs[:, 0]]
+            on_prefix = (coin < w.targets_on_prefix) & (first >= 0)
+            inside = ~on_prefix & (coin < w.targets_on_prefix + w.targets_in_image) & (image.size > 0)
+            run_target[inside] = pick[inside]
+            run_target[on_prefix] = first[on_prefix]
     return Static(vocab_map, runs, run_len, run_target)
 
 

@@ -78,6 +78,49 @@ def test_cache_hits_and_unmapped_stops_are_exercised(cuda_device):
     assert s.cache_hits > 50 and s.unmapped_stops > 5
 
 
+def _eq2_collision_counts(w, st, s, mp, vo):
+    """How many sequences of the step draw their extra token at a cached n-gram whose target
+    (a) has a direct pre-image of its own, (b) is the image of the run's first sub-token."""
+    image = np.zeros(w.v_p, bool)
+    image[st.vocab_map[st.vocab_map >= 0]] = True
+    m, n = mp.m.cpu().numpy(), vo.n_accepted.cpu().numpy()
+    tgt, sl, ss = mp.tgt_ids.cpu().numpy(), mp.span_len.cpu().numpy(), mp.span_start.cpu().numpy()
+    d = s.draft_ids.cpu().numpy()
+    inside = prefix = 0
+    for b in range(w.B):
+        j = int(n[b])
+        if j < int(m[b]) and sl[b, j] >= 2:
+            T = int(tgt[b, j])
+            on_prefix = int(st.vocab_map[d[b, ss[b, j]]]) == T
+            prefix += on_prefix
+            inside += bool(image[T]) and not on_prefix
+    return inside, prefix
+
+
+def test_eq2_collisions_cache_targets_inside_the_image(cuda_device):
+    """Eq. (2) when its cases collide: cached n-grams whose token has a direct pre-image, or is the
+    image of the run's own first sub-token. The residual of such a position must use the n-gram's
+    probability at that token (the oracle's reading, pinned by hand-worked vectors)."""
+    w = _small("eq2col", B=96, k_max=4, k_min=2, hit_prob=0.95, cache_entries=400, targets_in_image=0.4,
+               targets_on_prefix=0.4, rho=0.9, gen_seed=0xBEEF35)
+    st = synth.make_static(w)
+    ctx = parity.make_context(w, st, cuda_device)
+    cache = oracle.Cache(st.runs, st.run_len, st.run_target)
+    inside = prefix = 0
+    total = parity.Stats()
+    for step in range(6):
+        s = synth.make_step(w, st, step, device=cuda_device)
+        mp, vo, so = parity.gpu_step(ctx, s)
+        ref = parity.oracle_step(cache, st, w, s.to("cpu"), probe=so.out_token.cpu().numpy())
+        total.merge(parity.compare(mp, vo, so, ref, s.draft_len.cpu().numpy(), s.step,
+                                   s.seed.cpu().numpy().astype(np.uint64), bf16=True))
+        a, b = _eq2_collision_counts(w, st, s, mp, vo)
+        inside += a; prefix += b
+    ctx.close()
+    assert total.cache_hits > 100
+    assert inside >= 10 and prefix >= 10, (inside, prefix)
+
+
 @pytest.mark.parametrize("blocks_per_sm,tiles,pdl,dense", [(1, 1, 1, 1), (2, 2, 0, 2), (4, 7, 1, 3), (8, 1000, 0, 4),
                                                            (4, 5, 1, 0), (4, 3, 1, 5)])
 def test_every_split_of_a_row_gives_the_same_answer(cuda_device, blocks_per_sm, tiles, pdl, dense):

@@ -189,6 +189,71 @@ def test_eq2_hand_example_and_mass_conservation():
     assert qu.sum() == pytest.approx(float(q_row.astype(np.float64).sum()) - float(q_row[2]) + prod)
 
 
+def test_eq2_case_order_when_the_cases_collide():
+    """Eq. (2) is piecewise: the n-gram's token takes the n-gram's probability even when it
+    also has a direct pre-image, or when it is the image of the run's first sub-token."""
+    vals = {}
+    with open(os.path.join(GOLDEN, "eq2_hand_example.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            k, *v = line.split()
+            vals[k] = np.array([float(x) for x in v])
+    q_row = vals["q_row"].astype(np.float32)
+    prod = float(q_row[2]) * float(np.float32(vals["q_second"][0]))
+    vocab_map = np.arange(5, dtype=np.int32)
+    # (i) T = 3 has the direct pre-image 3
+    qf = oracle.full_mapping(q_row, vocab_map, 6, first_draft_id=2, length=2, ngram_token=3, ngram_prob=prod)
+    np.testing.assert_allclose(qf, vals["q_full_T_in_image"], atol=1e-7)
+    # (ii) T = 2 = map[d_1]
+    qf = oracle.full_mapping(q_row, vocab_map, 6, first_draft_id=2, length=2, ngram_token=2, ngram_prob=prod)
+    np.testing.assert_allclose(qf, vals["q_full_T_is_prefix"], atol=1e-7)
+
+
+def test_eq2_agrees_with_eq1_at_the_ngram_token_so_the_step_stays_lossless():
+    """The acceptance test of a merged position uses q'(T) of Eq. (1); the residual of the same
+    position uses q'(.) of Eq. (2). Speculative sampling returns p exactly only if both are the
+    same number at T: min(p, q') + max(0, p - q') = p. Checked through the oracle's own
+    translation (Eq. 1) and full mapping (Eq. 2) for targets outside the image, inside the
+    image, and equal to the image of the first sub-token."""
+    rng = np.random.default_rng(23)
+    V_q, V_p = 12, 20
+    vocab_map = np.full(V_q, -1, np.int32)
+    md = rng.permutation(V_q)[:8]
+    vocab_map[md] = rng.permutation(V_p)[:8]
+    image = set(int(t) for t in vocab_map if t >= 0)
+    outside = [t for t in range(V_p) if t not in image]
+    seen = set()
+    for trial in range(300):
+        L = int(rng.integers(2, 5))
+        run = rng.integers(0, V_q, size=L).astype(np.int32)
+        d1 = int(run[0])
+        kind = trial % 3
+        if kind == 0:
+            T = int(outside[rng.integers(0, len(outside))])
+        elif kind == 1:
+            T = int(vocab_map[md[rng.integers(0, len(md))]])
+        else:
+            if vocab_map[d1] < 0:
+                continue
+            T = int(vocab_map[d1])
+        seen.add((kind, T in image, vocab_map[d1] == T))
+        runs = np.full((1, 4), -1, np.int32); runs[0, :L] = run
+        cache = oracle.Cache(runs, np.array([L], np.int32), np.array([T], np.int32))
+        q_rows = rng.dirichlet(np.ones(V_q), size=L).astype(np.float32)
+        q_sel = np.array([q_rows[j, run[j]] for j in range(L)], np.float32)
+        tgt, qp, ss, sl, m, tail, hits = oracle.map_sequence(cache, vocab_map, run, q_sel)
+        assert m == 1 and hits == 1 and tgt[0] == T and sl[0] == L
+        qf = oracle.full_mapping(q_rows[0], vocab_map, V_p, d1, L, T, float(qp[0]))
+        assert qf[T] == qp[0]
+        p = rng.dirichlet(np.ones(V_p))
+        # emitted mass at T: accepted proposal + residual draw after a rejection of T
+        assert min(p[T], qp[0]) + max(0.0, p[T] - qf[T]) == pytest.approx(p[T], abs=1e-15)
+        if vocab_map[d1] >= 0 and vocab_map[d1] != T:
+            assert qf[vocab_map[d1]] == pytest.approx(float(q_rows[0, d1]) - qp[0], abs=1e-15)
+    assert (1, True, False) in seen and any(k[2] for k in seen)
+
+
 def test_full_mapping_through_a_random_partial_map():
     rng = np.random.default_rng(11)
     V_q, V_p = 50, 80
