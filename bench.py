@@ -64,8 +64,7 @@ def parse():
     ap.add_argument("--vocab-shards", type=int, default=0,
                     help="time one rank's kernels of the step with the target vocabulary split over this many GPUs")
     ap.add_argument("--shard-index", type=int, default=-1, help="the shard that is timed (default: the middle one)")
-    ap.add_argument("--verify-blocks-per-sm", type=int, default=0)
-    ap.add_argument("--verify-waves", type=int, default=0)
+    ap.add_argument("--verify-grid", type=int, default=0, help="thread blocks of the streaming kernel (0 = one per multiprocessor)")
     ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
     ap.add_argument("--sample-dense", type=int, default=-1, help="sampler pass 1: 0 automatic, 1 lists, 2..4 inverse map with that many tiles in flight, 5 pipelined pairs")
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches")
@@ -475,10 +474,11 @@ def main():
     ctx = od.Context(dev, w.v_q, w.v_p, w.B, w.k_max)
     ctx.set_vocab_map(st.vocab_map)
     ctx.cache_build(st.runs, st.run_len, st.run_target)
-    if a.verify_blocks_per_sm:
-        ctx.set_option("verify_blocks_per_sm", a.verify_blocks_per_sm)
-    if a.verify_waves:
-        ctx.set_option("verify_waves", a.verify_waves)
+    if a.verify_grid:
+        ctx.set_option("verify_grid", a.verify_grid)
+    # the pool's inputs are resident long before any timed launch: od_verify called on its own
+    # (the roofline graph) may read rows 0 before it waits for the launch in front
+    ctx.set_option("early_inputs", 1)
     if a.sample_tiles_per_warp:
         ctx.set_option("sample_tiles_per_warp", a.sample_tiles_per_warp)
     if a.sample_dense >= 0:

@@ -31,16 +31,23 @@
  *     must be ordered (one stream, or explicit dependencies). Use one context
  *     per concurrent stream, and make the calls of one step on one context.
  *   - With option "pdl" = 1 (the default) the step kernels are launched with
- *     programmatic stream serialization and start work on their INPUTS before
- *     the launch in front of them in the stream has finished: od_verify reads
- *     logits and temperatures early, od_sample_residual the outputs of
- *     od_map_proposals (not when the call in front of it on its context was
- *     od_map_proposals itself). So the step's inputs (draft ids, lengths and
- *     probabilities, logits, temperatures, seeds) must be complete before the
- *     launch that precedes the step's first call is enqueued; a producer that
- *     is itself the preceding launch is fine if it is an ordinary kernel launch
- *     (it has finished by the time a dependent kernel starts). "pdl" = 0 gives
- *     plain stream order.
+ *     programmatic stream serialization: a kernel may become resident while
+ *     the launch in front of it in the stream still runs, and executes
+ *     griddepcontrol.wait before it touches anything that launch may write.
+ *     What a kernel reads BEFORE its wait is only what the library itself can
+ *     prove complete: outputs of a library kernel that finished before the
+ *     kernel in front was allowed to start. Inputs of the caller (logits,
+ *     temperatures, seeds, draft ids and probabilities) are read before the
+ *     wait in two cases only: inside od_step / od_step_host, where the
+ *     translation kernel is the launch in front of the streaming kernel and has
+ *     itself waited for everything earlier in the stream before letting it
+ *     start; and in od_verify when the caller has set option "early_inputs" = 1,
+ *     which is the caller's promise that the step's inputs were complete before
+ *     the launch that precedes the call was enqueued (a producer two launches
+ *     back, or data resident since an earlier synchronisation). A producer that
+ *     is the launch directly in front of od_verify (the target model's output
+ *     layer, say) is always safe with the default "early_inputs" = 0.
+ *     "pdl" = 0 gives plain stream order.
  *   - Positions: arrays indexed [B, K_max] hold K_max entries per sequence,
  *     of which the first K_b (inputs) or m_b (outputs) are meaningful.
  *   - Random numbers: Philox4x32-10 (Salmon et al., SC'11) with key = the
@@ -190,16 +197,14 @@ int32_t od_cache_trim(od_ctx *ctx, void *stream);
 int32_t od_cache_dump(od_ctx *ctx, int64_t max_out, int32_t *runs, int32_t *len,
                       int32_t *target, uint32_t *stamp, uint32_t *freq, int64_t *n_out);
 
-/* Tuning knobs, mainly for experiments. Names: "verify_blocks_per_sm" (thread
- * blocks of od_verify per multiprocessor, 1..8, 0 = automatic),
- * "sample_tiles_per_warp" (256-id tiles one warp of od_sample_residual sums,
- * 0 = automatic), "sample_dense" (how the first pass of od_sample_residual finds
- * the drafter's probability of a target id: 1 = through per-tile lists of the mapped
- * ids, 2..4 = through the inverse map with that many tiles in flight per warp,
- * 5 = through the inverse map, pairs of tiles software-pipelined, 0 = automatic),
- * "pdl" (1 = launch the step kernels with programmatic stream
- * serialization so that a kernel's prologue overlaps its predecessor's tail,
- * the default; 0 = plain stream order). Unknown name: INVALID_ARG. */
+/* Options. Names: "pdl" (1 = launch the step kernels with programmatic stream
+ * serialization so that a kernel's prologue overlaps its predecessor's tail, the
+ * default; 0 = plain stream order), "early_inputs" (1 = od_verify and
+ * od_verify_shard_stats may read logits and temperatures before they wait for the
+ * launch in front of them, see the conventions above; default 0),
+ * "verify_grid" (thread blocks of od_verify's streaming kernel, 0 = one per
+ * multiprocessor, the default), "sample_tiles_per_warp" (256-id tiles one warp of
+ * od_sample_residual sums, 0 = automatic). Unknown name: INVALID_ARG. */
 int32_t od_set_option(od_ctx *ctx, const char *name, int64_t value);
 
 /* ---- the step ----------------------------------------------------------- */
@@ -282,6 +287,26 @@ int32_t od_sample_residual(od_ctx *ctx, int32_t B, int32_t K_max,
                            const uint64_t *seed, uint64_t step,
                            int32_t *out_token, float *resid_mass,
                            uint32_t *sample_flags, void *stream);
+
+/* Steps 1-3 in one call (Algorithm 1 from the translation line to the free-token
+ * line): exactly od_map_proposals, od_verify and od_sample_residual on the same
+ * arguments, enqueued back to back on `stream`. Besides saving two calls, this is
+ * the form in which the library knows its own launch order, so the streaming
+ * kernel may start on rows 0 of the logits while the translation kernel still
+ * runs, with no promise needed from the caller (see "pdl" in the conventions).
+ * All pointers are device pointers owned by the caller; inputs and outputs as
+ * documented for the three calls (counters may be NULL). Asynchronous; allocates
+ * nothing; errors as for the three calls, checked before the first launch. */
+int32_t od_step(od_ctx *ctx, int32_t B, int32_t K_max, const int32_t *draft_ids,
+                const int32_t *draft_len, const float *q_sel, const float *q_rows,
+                const void *logits, int32_t logit_dtype, int64_t row_stride,
+                int64_t seq_stride, const float *temperature, const uint64_t *seed,
+                uint64_t step, int32_t *tgt_ids, float *q_prime, int32_t *span_start,
+                int32_t *span_len, int32_t *m, uint8_t *tail_kind, uint32_t *counters,
+                float *row_max, float *row_sum, float *p_sel, float *ratio,
+                int32_t *n_accepted, int32_t *n_draft_accepted, uint32_t *verify_flags,
+                int32_t *out_token, float *resid_mass, uint32_t *sample_flags,
+                void *stream);
 
 /* Hybrid cross-vocabulary distillation loss (Section 3.2, Eq. (3)) of the proposals
  * of one verification step, per draft position j, and its gradient with respect to
@@ -485,8 +510,8 @@ int32_t od_sample_shard_pick(od_ctx *ctx, int32_t B, int32_t K_max, int32_t n_sh
 /* ---- misc ---------------------------------------------------------------- */
 
 /* Launch shape of the last od_verify / od_sample_residual call on this context
- * (for benchmarks). which: 0 = verify grid size, 1 = 512-byte units of row 0
- * data per warp, 2 = sample grid size, 3 = sample tiles per warp. */
+ * (for benchmarks). which: 0 = verify grid size, 1 = 512-byte units of row 0 data per
+ * thread block, 2 = sample grid size, 3 = sample tiles per warp. */
 int64_t od_last_launch_info(const od_ctx *ctx, int32_t which);
 
 const char *od_status_string(int32_t status);

@@ -30,7 +30,7 @@ OD_MAX_K = 16
 OD_NOALLOC_MAX_ROWS = 1024
 
 EXPORTS = ["od_create", "od_destroy", "od_set_vocab_map", "od_cache_build", "od_set_option",
-           "od_map_proposals", "od_verify", "od_sample_residual", "od_host_step_reserve",
+           "od_map_proposals", "od_verify", "od_sample_residual", "od_step", "od_host_step_reserve",
            "od_step_host", "od_verify_noalloc", "od_exit_rule", "od_cache_configure", "od_cache_set_clock",
            "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_distill_loss",
            "od_verify_shard_stats", "od_verify_shard_finish", "od_sample_shard_mass", "od_sample_shard_pick",
@@ -66,6 +66,7 @@ def lib():
         L.od_verify.argtypes = [vp, i32, i32, vp, i32, i64, i64] + [vp] * 6 + [u64] + [vp] * 7 + [vp]
         L.od_sample_residual.argtypes = ([vp, i32, i32, vp, i32, i64, i64] + [vp] * 13 + [u64]
                                          + [vp] * 3 + [vp])
+        L.od_step.argtypes = ([vp, i32, i32] + [vp] * 5 + [i32, i64, i64, vp, vp, u64] + [vp] * 17 + [vp])
         L.od_verify_noalloc.argtypes = [i32, i32, i32, vp, i32, i64, i64] + [vp] * 6 + [u64] + [vp] * 7 + [vp]
         L.od_exit_rule.argtypes = [vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp]
         L.od_distill_loss.argtypes = ([vp, i32, i32] + [vp] * 7 + [i32, i64, i64] + [vp] * 4
@@ -370,6 +371,31 @@ def od_sample_residual(ctx: Context, logits, vo: VerifyOut, q_rows, draft_ids, m
         _dp(out.out_token, i32, d), _dp(out.resid_mass, f32, d), _dp(out.flags, i32, d),
         _stream(d)), "od_sample_residual")
     return out
+
+
+def od_step(ctx: Context, s_draft_ids, s_draft_len, s_q_sel, s_q_rows, logits, temperature, seed, step: int,
+            mp: Optional[MapOut] = None, vo: Optional[VerifyOut] = None, so: Optional[SampleOut] = None):
+    """Steps 1-3 in one call on device tensors: (MapOut, VerifyOut, SampleOut)."""
+    B, K = s_draft_ids.shape
+    mp = mp or alloc_map_out(ctx, B, K)
+    vo = vo or alloc_verify_out(ctx, B, K)
+    so = so or alloc_sample_out(ctx, B)
+    d, i32, f32 = ctx.device, torch.int32, torch.float32
+    rs, ss = _strides(logits, B, K, ctx.target_vocab)
+    if logits.device != d:
+        raise ValueError("logits on another device")
+    if tuple(s_q_rows.shape) != (B, K, ctx.draft_vocab):
+        raise ValueError("q_rows must be [B, K, V_q]")
+    _check(lib().od_step(
+        ctx.handle, B, K, _dp(s_draft_ids, i32, d), _dp(s_draft_len, i32, d), _dp(s_q_sel, f32, d),
+        _dp(s_q_rows, f32, d), C.c_void_p(logits.data_ptr()), logit_dtype_code(logits), rs, ss,
+        _dp(temperature, f32, d), _dp(seed, torch.int64, d), C.c_uint64(step & (2**64 - 1)),
+        _dp(mp.tgt_ids, i32, d), _dp(mp.q_prime, f32, d), _dp(mp.span_start, i32, d), _dp(mp.span_len, i32, d),
+        _dp(mp.m, i32, d), _dp(mp.tail_kind, torch.uint8, d), _dp(mp.counters, i32, d),
+        _dp(vo.row_max, f32, d), _dp(vo.row_sum, f32, d), _dp(vo.p_sel, f32, d), _dp(vo.ratio, f32, d),
+        _dp(vo.n_accepted, i32, d), _dp(vo.n_draft_accepted, i32, d), _dp(vo.flags, i32, d),
+        _dp(so.out_token, i32, d), _dp(so.resid_mass, f32, d), _dp(so.flags, i32, d), _stream(d)), "od_step")
+    return mp, vo, so
 
 
 # ---- the step with the target vocabulary split over GPUs (one call per phase) ----

@@ -266,8 +266,8 @@ int32_t od_cache_build(od_ctx *c, const int32_t *host_runs, const int32_t *host_
 int32_t od_set_option(od_ctx *c, const char *name, int64_t value)
 {
     if (!c || !name || value < 0) return OD_ERR_INVALID_ARG;
-    if (!strcmp(name, "verify_blocks_per_sm")) { c->opt_verify_blocks_per_sm = value; return OD_OK; }
-    if (!strcmp(name, "verify_waves")) { c->opt_verify_waves = value; return OD_OK; }
+    if (!strcmp(name, "verify_grid")) { c->opt_verify_grid = value; return OD_OK; }
+    if (!strcmp(name, "early_inputs")) { c->opt_early_inputs = value != 0; return OD_OK; }
     if (!strcmp(name, "sample_tiles_per_warp")) { c->opt_sample_tiles_per_warp = value; return OD_OK; }
     if (!strcmp(name, "pdl")) { c->opt_pdl = value != 0; return OD_OK; }
     if (!strcmp(name, "sample_dense")) {
@@ -311,6 +311,7 @@ int32_t od_verify(od_ctx *c, int32_t B, int32_t K_max, const void *logits, int32
         return OD_ERR_INVALID_ARG;
     DeviceGuard g(c->device);
     if (!g.ok) return OD_ERR_CUDA;
+    c->verify_early = c->opt_early_inputs != 0;
     OD_CUDA(od_launch_verify(c, B, K_max, logits, logit_dtype, row_stride, seq_stride, tgt_ids,
                              q_prime, span_len, m, temperature, seed, step, row_max, row_sum,
                              p_sel, ratio, n_accepted, n_draft_accepted, verify_flags,
@@ -345,6 +346,41 @@ int32_t od_sample_residual(od_ctx *c, int32_t B, int32_t K_max, const void *logi
     return OD_OK;
 }
 
+int32_t od_step(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids, const int32_t *draft_len,
+                const float *q_sel, const float *q_rows, const void *logits, int32_t logit_dtype,
+                int64_t row_stride, int64_t seq_stride, const float *temperature, const uint64_t *seed,
+                uint64_t step, int32_t *tgt_ids, float *q_prime, int32_t *span_start, int32_t *span_len,
+                int32_t *m, uint8_t *tail_kind, uint32_t *counters, float *row_max, float *row_sum,
+                float *p_sel, float *ratio, int32_t *n_accepted, int32_t *n_draft_accepted,
+                uint32_t *verify_flags, int32_t *out_token, float *resid_mass, uint32_t *sample_flags,
+                void *stream)
+{
+    int32_t st = check_step_common(c, B, K_max);
+    if (st != OD_OK) return st;
+    st = check_logits(c, logits, logit_dtype, row_stride, seq_stride, K_max);
+    if (st != OD_OK) return st;
+    if (!draft_ids || !draft_len || !q_sel || !q_rows || !temperature || !seed || !tgt_ids || !q_prime ||
+        !span_start || !span_len || !m || !tail_kind || !row_max || !row_sum || !p_sel || !ratio ||
+        !n_accepted || !n_draft_accepted || !verify_flags || !out_token || !resid_mass || !sample_flags)
+        return OD_ERR_INVALID_ARG;
+    DeviceGuard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    OD_CUDA(od_launch_map(c, B, K_max, draft_ids, draft_len, q_sel, tgt_ids, q_prime, span_start, span_len, m,
+                          tail_kind, counters, s));
+    // The translation kernel waits for everything in front of it before it lets the next
+    // kernel start, so whatever wrote the logits has finished by the time a block of the
+    // stream kernel runs: rows 0 may be read before that kernel's own wait.
+    c->verify_early = true;
+    OD_CUDA(od_launch_verify(c, B, K_max, logits, logit_dtype, row_stride, seq_stride, tgt_ids, q_prime,
+                             span_len, m, temperature, seed, step, row_max, row_sum, p_sel, ratio,
+                             n_accepted, n_draft_accepted, verify_flags, s));
+    OD_CUDA(od_launch_sample(c, B, K_max, logits, logit_dtype, row_stride, seq_stride, row_max, row_sum,
+                             q_rows, draft_ids, tgt_ids, q_prime, span_start, span_len, m, tail_kind,
+                             n_accepted, temperature, seed, step, out_token, resid_mass, sample_flags, s));
+    return OD_OK;
+}
+
 int32_t od_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo, int32_t shard_len,
                               const void *logits, int32_t logit_dtype, int64_t row_stride,
                               int64_t seq_stride, const int32_t *tgt_ids, const int32_t *m,
@@ -360,6 +396,7 @@ int32_t od_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, int32_t shard
     if (!aligned16(stats)) return OD_ERR_ALIGNMENT;
     DeviceGuard g(c->device);
     if (!g.ok) return OD_ERR_CUDA;
+    c->verify_early = c->opt_early_inputs != 0;
     OD_CUDA(od_launch_verify_shard_stats(c, B, K_max, shard_lo, shard_len, logits, logit_dtype, row_stride,
                                          seq_stride, tgt_ids, m, temperature, stats, (cudaStream_t)stream));
     return OD_OK;
@@ -577,6 +614,7 @@ int32_t od_step_host(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_i
     }
     OD_CUDA(od_launch_map(c, B, K_max, c->s_draft_ids, c->s_draft_len, c->s_q_sel, c->s_tgt_ids,
                           c->s_q_prime, c->s_span_start, c->s_span_len, c->s_m, c->s_tail, nullptr, s));
+    c->verify_early = true;     // the translation kernel is the launch in front: see od_step
     OD_CUDA(od_launch_verify(c, B, K_max, c->s_logits, logit_dtype, row_stride, seq_stride,
                              c->s_tgt_ids, c->s_q_prime, c->s_span_len, c->s_m, c->s_temperature,
                              c->s_seed, step, c->s_row_max, c->s_row_sum, c->s_p_sel, c->s_ratio,

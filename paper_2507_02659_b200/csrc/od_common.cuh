@@ -59,11 +59,14 @@ struct od_ctx {
     int32_t tiles_per_row;
 
     // options
-    int64_t opt_verify_blocks_per_sm;
-    int64_t opt_verify_waves;       // grid = waves x the resident capacity (experiments)
+    int64_t opt_verify_grid;        // blocks of the stream kernel (0 = one per multiprocessor)
+    int64_t opt_early_inputs;       // od_verify may read logits and temperatures before griddepcontrol.wait
     int64_t opt_sample_tiles_per_warp;
     int64_t opt_sample_dense;       // pass 1 of the sampler: 0 = automatic, 1 = lists, 2..4 = inverse map, that many tiles in flight, 5 = pipelined pairs
     int64_t opt_pdl;                // launch with programmatic stream serialization
+
+    // set by the entry points for the verify launch that follows: space A may be streamed early
+    bool verify_early;
 
     // the last launch on this context was the translation kernel, which lets the next
     // kernel start before its own outputs exist (see od_sample.cu)
@@ -99,6 +102,7 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              float *row_max, float *row_sum, float *p_sel, float *ratio,
                              int32_t *n_accepted, int32_t *n_draft_accepted,
                              uint32_t *flags, cudaStream_t s);
+
 
 cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
                              int32_t dtype, int64_t row_stride, int64_t seq_stride,

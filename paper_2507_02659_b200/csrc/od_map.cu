@@ -6,7 +6,8 @@
 // cache is an open-addressing table of 32-slot groups, a probe reads one group
 // with one coalesced 256-byte load (lane <-> slot) and resolves it with two
 // ballots (key match / empty slot). The first probes of the three lengths are
-// issued together so their latencies overlap. After a block barrier one thread
+// issued together, each with the values of its group, so their latencies overlap
+// and a hit in the first group costs one memory round trip. After a block barrier one thread
 // walks the proposal left to right, longest hit first, then the direct map,
 // and writes the mapped proposal. Integer work throughout, except the product
 // of at most four fp32 draft probabilities.
@@ -14,20 +15,25 @@
 
 namespace {
 
-// returns the slot that holds `key`, or -1
-__device__ __forceinline__ int32_t probe_continue(const uint64_t *__restrict__ keys,
+// Resolves a lookup whose first group g is already loaded (keys in k_lane, values in
+// v_lane): the slot that holds `key` and its value, or -1. Walks at most ngroups groups,
+// so it ends on any table contents.
+__device__ __forceinline__ int32_t probe_continue(const uint64_t *__restrict__ keys, const int32_t *__restrict__ vals,
                                                   uint64_t ngroups, uint64_t key, uint64_t g,
-                                                  uint64_t k_lane, int lane)
+                                                  uint64_t k_lane, int32_t v_lane, int lane, int32_t *value)
 {
-    // resolves a lookup whose first group (already loaded into k_lane) is g;
-    // walks at most ngroups groups, so it ends on any table contents
     for (uint64_t step = 0; step < ngroups; ++step) {
         unsigned match = __ballot_sync(0xFFFFFFFFu, k_lane == key);
-        if (match) return (int32_t)(g * OD_GROUP + (__ffs(match) - 1));
+        if (match) {
+            const int src = __ffs(match) - 1;
+            *value = __shfl_sync(0xFFFFFFFFu, v_lane, src);
+            return (int32_t)(g * OD_GROUP + src);
+        }
         unsigned empty = __ballot_sync(0xFFFFFFFFu, k_lane == 0ULL);
         if (empty) return -1;
         g = (g + 1) & (ngroups - 1);
         k_lane = __ldg(keys + g * OD_GROUP + lane);
+        v_lane = __ldcg(vals + g * OD_GROUP + lane);
     }
     return -1;
 }
@@ -75,6 +81,7 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
         if (cap > 0) {
             const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
             uint64_t key[OD_NGRAM_MAX + 1], grp[OD_NGRAM_MAX + 1], kl[OD_NGRAM_MAX + 1];
+            int32_t vl[OD_NGRAM_MAX + 1];
             bool valid[OD_NGRAM_MAX + 1];
             // ids of a run must lie in the draft vocabulary; the run must fit
             bool ok = true;
@@ -89,14 +96,19 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
                 grp[L] = od_hash64(k) & (ngroups - 1);
             }
 #pragma unroll
-            for (int L = 2; L <= OD_NGRAM_MAX; ++L)
+            for (int L = 2; L <= OD_NGRAM_MAX; ++L) {
                 kl[L] = valid[L] ? __ldg(keys + grp[L] * OD_GROUP + lane) : 0ULL;
+                // the values of the group come with its keys, so a hit costs one round trip
+                // (a concurrent batch insert writes an entry's value last: read it past L1)
+                vl[L] = valid[L] ? __ldcg(vals + grp[L] * OD_GROUP + lane) : -1;
+            }
 #pragma unroll
             for (int L = 2; L <= OD_NGRAM_MAX; ++L)
                 if (valid[L]) {
-                    slot[L] = probe_continue(keys, ngroups, key[L], grp[L], kl[L], lane);
-                    // an entry whose value is not set yet does not exist (a concurrent batch insert writes it last)
-                    if (slot[L] >= 0) hit[L] = __ldg(vals + slot[L]);
+                    int32_t value = -1;
+                    slot[L] = probe_continue(keys, vals, ngroups, key[L], grp[L], kl[L], vl[L], lane, &value);
+                    // an entry whose value is not set yet does not exist
+                    if (slot[L] >= 0) hit[L] = value;
                 }
         }
         if (lane == 0) {

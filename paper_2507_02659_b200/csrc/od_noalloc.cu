@@ -87,6 +87,7 @@ extern "C" int32_t od_verify_noalloc(int32_t target_vocab, int32_t B, int32_t K_
     c.sm_count = dev.sm_count;
     c.d_partials = dev.partials;
     c.opt_pdl = 1;
+    c.verify_early = false;     // nothing is known about the launch in front: wait before reading
     if (od_launch_verify(&c, B, K_max, logits, logit_dtype, row_stride, seq_stride, tgt_ids, q_prime,
                          span_len, m, temperature, seed, step, row_max, row_sum, p_sel, ratio,
                          n_accepted, n_draft_accepted, verify_flags, (cudaStream_t)stream) != cudaSuccess)

@@ -11,10 +11,11 @@
 // bytes of a row; a row has W units; the rows to read are laid end to end in
 // two flat index spaces and every block takes one contiguous span of each:
 //   space A  row 0 of every sequence. It is always read and its split needs
-//            nothing from the device, so a block works through its span
-//            before it waits for the translation kernel (programmatic
-//            dependent launch): that kernel, and the previous launch's decide
-//            kernel, are hidden behind useful traffic;
+//            nothing from the device, so when the library knows that the
+//            logits are complete (see `a_early`) a block works through its
+//            span before it waits for the launch in front (programmatic
+//            dependent launch): the translation kernel, or the previous
+//            launch's decide kernel, is hidden behind useful traffic;
 //   space B  rows 1..m_b, split by the prefix sums of m, which every block
 //            rebuilds in shared memory (at most 2048 sequences per launch).
 // A span is cut at row ends into segments; every warp of the block reduces its
@@ -68,7 +69,8 @@ struct VerifyArgs {
     int32_t n_chunks;                   // blocks of the stream grid
     int32_t span_min;                   // keeps a row within OD_VERIFY_SEG_MAX / WARPS block segments
     int32_t span_a;                     // units of space A per block
-    int32_t a_early;                    // 1: a block's span of space A has at most A_PARK segments
+    int32_t a_early;                    // 1: space A is streamed before griddepcontrol.wait (the caller allows
+                                        // it and a block's span of space A has at most A_PARK segments)
     const int32_t *tgt_ids;
     const float *q_prime;
     const int32_t *span_len;
@@ -325,10 +327,11 @@ od_verify_stream_kernel(const VerifyArgs a)
     const uint32_t W = (uint32_t)a.W;
 
     // ---- space A (row 0 of every sequence). Nothing here depends on the translation
-    // kernel (logits and temperatures are inputs of the step), so under programmatic
-    // dependent launch this phase runs while that kernel is still at work. Its partials
-    // wait in shared memory: the scratch in global memory may still be read by the
-    // previous launch's decide kernel until griddepcontrol.wait returns.
+    // kernel (logits and temperatures are inputs of the step), so where those inputs are
+    // known to be complete (a_early) this phase runs, under programmatic dependent launch,
+    // while the launch in front is still at work. Its partials wait in shared memory: the
+    // scratch in global memory may still be read by the previous launch's decide kernel
+    // until griddepcontrol.wait returns.
     const uint32_t a_tot = (uint32_t)a.B * W;
     uint32_t a_lo = g * (uint32_t)a.span_a;
     if (a_lo > a_tot) a_lo = a_tot;
@@ -632,7 +635,8 @@ cudaError_t launch(Kern kern, unsigned grid, unsigned block, cudaStream_t s, boo
 }  // namespace
 
 // Launch plan of the stream kernel for `nb` sequences whose rows hold `v_len` elements.
-static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_len, int32_t dtype, VerifyArgs &a)
+static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_len, int32_t dtype, bool early,
+                        VerifyArgs &a)
 {
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
     const int64_t row_bytes = (int64_t)v_len * esz;
@@ -640,11 +644,9 @@ static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_le
     // a row is cut into at most OD_VERIFY_SEG_MAX / WARPS block segments (one partial per warp each)
     constexpr int MAX_BLOCK_SEGS = OD_VERIFY_SEG_MAX / WARPS;
     const int32_t span_min = (W + MAX_BLOCK_SEGS - 2) / (MAX_BLOCK_SEGS - 1);
-    int64_t blocks_per_sm = c->opt_verify_blocks_per_sm > 0 ? c->opt_verify_blocks_per_sm : OD_VERIFY_BLOCKS_PER_SM;
-    if (blocks_per_sm > OD_VERIFY_BLOCKS_PER_SM) blocks_per_sm = OD_VERIFY_BLOCKS_PER_SM;
-    // no more blocks than the most this slice can need
+    // one resident wave, and no more blocks than the most this slice can need
     const int64_t max_units = (int64_t)nb * (K_max + 1) * W;
-    int64_t grid = (int64_t)c->sm_count * blocks_per_sm * (c->opt_verify_waves > 0 ? c->opt_verify_waves : 1);
+    int64_t grid = c->opt_verify_grid > 0 ? c->opt_verify_grid : (int64_t)c->sm_count * OD_VERIFY_BLOCKS_PER_SM;
     const int64_t need = max_units / span_min + 1;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
@@ -653,7 +655,7 @@ static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_le
     int64_t span_a = ((int64_t)nb * W + grid - 1) / grid;
     if (span_a < span_min) span_a = span_min;
     a.span_a = (int32_t)span_a;
-    a.a_early = span_a / W + 2 <= A_PARK;
+    a.a_early = early && span_a / W + 2 <= A_PARK;
 }
 
 // batches beyond the shared-memory prefix table go in slices; a slice's flat
@@ -681,7 +683,7 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
     for (int32_t b0 = 0; b0 < B; b0 += slice) {
         const int32_t nb = B - b0 < slice ? B - b0 : slice;
         VerifyArgs a = {};
-        plan_stream(c, nb, K_max, c->v_p, dtype, a);
+        plan_stream(c, nb, K_max, c->v_p, dtype, c->verify_early, a);
         a.logits = (const char *)logits + (size_t)b0 * seq_stride * esz;
         a.row_stride = row_stride; a.seq_stride = seq_stride;
         a.tgt_ids = tgt_ids + (size_t)b0 * K_max; a.q_prime = q_prime + (size_t)b0 * K_max;
@@ -723,7 +725,7 @@ cudaError_t od_launch_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, in
     for (int32_t b0 = 0; b0 < B; b0 += slice) {
         const int32_t nb = B - b0 < slice ? B - b0 : slice;
         VerifyArgs a = {};
-        plan_stream(c, nb, K_max, shard_len, dtype, a);
+        plan_stream(c, nb, K_max, shard_len, dtype, c->verify_early, a);
         a.logits = (const char *)logits + (size_t)b0 * seq_stride * esz;
         a.row_stride = row_stride; a.seq_stride = seq_stride;
         a.tgt_ids = tgt_ids + (size_t)b0 * K_max; a.m = m + b0;

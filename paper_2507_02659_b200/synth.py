@@ -50,6 +50,9 @@ class Workload:
     # collisions between the cases of Eq. (2):
     targets_in_image: float = 0.0    # share of entries whose target has a direct pre-image
     targets_on_prefix: float = 0.0   # share whose target is the image of the run's first id
+    # Added to the draft logits of a planted run's ids, so that the drafter itself finds the run
+    # likely (q' of the merged token is then large enough for the token to be rejected sometimes):
+    plant_boost: float = 0.0
 
 
 def paper_config(i: int) -> Workload:
@@ -253,6 +256,11 @@ def make_step(w: Workload, st: Static, step: int, device="cpu",
         nb = hi - lo
         z_q = torch.randn(nb, K, Vq, generator=g, device=dev, dtype=torch.float32) * w.sigma
         T = temps[lo:hi].view(nb, 1, 1)
+        if w.plant_boost > 0:
+            for b in range(lo, hi):
+                e = int(plant[b])
+                for j in range(int(st.run_len[e]) if e >= 0 else 0):
+                    z_q[b - lo, int(plant_off[b]) + j, int(st.runs[e, j])] += w.plant_boost
         qr = torch.softmax(((z_q - shift) / T).double(), dim=-1).float()
         q_rows[lo:hi] = qr
         ids = torch.multinomial(qr.view(nb * K, Vq), 1, generator=g).view(nb, K)

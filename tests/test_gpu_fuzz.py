@@ -28,7 +28,12 @@ def _random_workload(rng, i):
         mapped_frac=frac, cache_entries=entries, hit_prob=float(rng.uniform(0, 1)) if entries else 0.0,
         logit_kind=["corr", "noise", "zipf"][int(rng.integers(0, 3))], rho=0.9,
         temperatures=tuple(float(t) for t in rng.choice([0.3, 0.5, 0.7, 1.0, 1.5], size=3)),
-        per_seq_seed=True, gen_seed=0xF00D00 + i, unmapped_shift=float(rng.uniform(0, 4)), sigma=2.0)
+        per_seq_seed=True, gen_seed=0xF00D00 + i, unmapped_shift=float(rng.uniform(0, 4)), sigma=2.0,
+        # every third case: cached n-grams whose token collides with the direct map (the cases of
+        # Eq. (2) overlap), made likely enough under the drafter to be rejected now and then
+        targets_in_image=0.3 if i % 3 == 0 and entries else 0.0,
+        targets_on_prefix=0.3 if i % 3 == 0 and entries else 0.0,
+        plant_boost=8.0 if i % 3 == 0 and entries else 0.0)
 
 
 @pytest.mark.parametrize("i", range(24))

@@ -66,6 +66,30 @@ def test_sharded_step_matches_the_oracle(cuda_device, n_shards, dtype, copy):
     ctx.close()
 
 
+def test_sharded_step_with_colliding_cases_of_eq2(cuda_device):
+    """Cached n-grams whose token has a direct pre-image, or is the image of the run's own first
+    sub-token, rejected often enough that the sharded residual draw meets them."""
+    w = _workload("vs_eq2", B=64, k_max=4, k_min=2, v_q=600, v_p=1000, cache_entries=400, hit_prob=0.95,
+                  logit_kind="zipf", targets_in_image=0.4, targets_on_prefix=0.4, plant_boost=8.0,
+                  gen_seed=0xBEEF9E)
+    st = synth.make_static(w)
+    ctx = parity.make_context(w, st, cuda_device)
+    cache = oracle.Cache(st.runs, st.run_len, st.run_target)
+    image = np.zeros(w.v_p, bool)
+    image[st.vocab_map[st.vocab_map >= 0]] = True
+    at_ngram_in_image = 0
+    for step in range(4):
+        s = synth.make_step(w, st, step, device=cuda_device)
+        _, (mp, vo, so) = _sharded_check(ctx, cache, st, w, s, 3)
+        m, n = mp.m.cpu().numpy(), vo.n_accepted.cpu().numpy()
+        tgt, sl = mp.tgt_ids.cpu().numpy(), mp.span_len.cpu().numpy()
+        for b in range(w.B):
+            j = int(n[b])
+            at_ngram_in_image += j < int(m[b]) and sl[b, j] >= 2 and bool(image[tgt[b, j]])
+    assert at_ngram_in_image >= 20
+    ctx.close()
+
+
 def test_one_shard_is_bit_identical_to_the_unsharded_calls(cuda_device):
     w = _workload("vs1bits", B=40, v_p=9000)
     st = synth.make_static(w)
