@@ -66,7 +66,6 @@ def parse():
     ap.add_argument("--shard-index", type=int, default=-1, help="the shard that is timed (default: the middle one)")
     ap.add_argument("--verify-grid", type=int, default=0, help="thread blocks of the streaming kernel (0 = one per multiprocessor)")
     ap.add_argument("--sample-tiles-per-warp", type=int, default=0)
-    ap.add_argument("--sample-dense", type=int, default=-1, help="sampler pass 1: 0 automatic, 1 lists, 2..4 inverse map with that many tiles in flight, 5 pipelined pairs")
     ap.add_argument("--no-pdl", action="store_true", help="plain stream-ordered launches")
     return ap.parse_args()
 
@@ -481,8 +480,6 @@ def main():
     ctx.set_option("early_inputs", 1)
     if a.sample_tiles_per_warp:
         ctx.set_option("sample_tiles_per_warp", a.sample_tiles_per_warp)
-    if a.sample_dense >= 0:
-        ctx.set_option("sample_dense", a.sample_dense)
     if a.no_pdl:
         ctx.set_option("pdl", 0)
 

@@ -125,7 +125,10 @@ enum od_counter {
  * `draft_vocab` ids and a target vocabulary of `target_vocab` ids, for
  * batches of at most `max_batch` sequences with at most `max_k`
  * (1..OD_MAX_K) proposed tokens each. Allocates the device-side scratch
- * (tickets, partial row statistics, tile sums) once; synchronous. */
+ * (tickets, partial row statistics, tile sums) once; synchronous.
+ * target_vocab is bounded by what od_sample_residual keeps in shared memory
+ * (8 bytes per 256 ids, at most 200 KB: 6,553,600 ids); larger vocabularies
+ * are refused with OD_ERR_UNSUPPORTED. */
 int32_t od_create(od_ctx **ctx, int32_t device, int32_t draft_vocab,
                   int32_t target_vocab, int32_t max_batch, int32_t max_k);
 

@@ -45,7 +45,7 @@ int32_t dev_alloc(T **p, size_t n)
 void free_all(od_ctx *c)
 {
     od_cache_free_dynamic(c);
-    void *ptrs[] = {c->d_vocab_map, c->d_inv_map, c->d_mapped_t, c->d_mapped_d, c->d_keys, c->d_vals, c->d_partials,
+    void *ptrs[] = {c->d_vocab_map, c->d_inv_map, c->d_keys, c->d_vals, c->d_partials,
                     c->d_tile_sums,
                     c->d_samp_ticket, c->s_logits, c->s_q_rows, c->s_q_sel, c->s_temperature,
                     c->s_draft_ids, c->s_draft_len, c->s_seed, c->s_tgt_ids, c->s_span_start,
@@ -125,6 +125,15 @@ int32_t od_create(od_ctx **ctx, int32_t device, int32_t draft_vocab, int32_t tar
     }
     c->opt_pdl = 1;
     c->tiles_per_row = (target_vocab + OD_SAMPLE_TILE - 1) / OD_SAMPLE_TILE;
+    // the sampler keeps a row's tile values in shared memory: that bounds the target vocabulary
+    if (od_sample_smem_bytes(c->tiles_per_row) > OD_SAMPLE_SMEM_MAX) {
+        delete c;
+        return OD_ERR_UNSUPPORTED;
+    }
+    if (od_sample_prepare_device(od_sample_smem_bytes(c->tiles_per_row)) != cudaSuccess) {
+        delete c;
+        return OD_ERR_CUDA;
+    }
     // od_verify scratch serves one launch: at most OD_VERIFY_MAX_B sequences
     const size_t vb = max_batch < OD_VERIFY_MAX_B ? max_batch : OD_VERIFY_MAX_B;
     const size_t rows = vb * (max_k + 1);
@@ -173,31 +182,6 @@ int32_t od_set_vocab_map(od_ctx *c, const int32_t *host_map)
     for (int32_t d = 0; d < c->v_q; ++d) fwd[d] = host_map[d] < 0 ? -1 : host_map[d];
     OD_CUDA(cudaMemcpy(c->d_vocab_map, fwd.data(), fwd.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
     OD_CUDA(cudaMemcpy(c->d_inv_map, inv.data(), inv.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
-    // the same inverse map as one fixed-width list per tile of target ids (for the residual sampler)
-    const size_t ntiles = (size_t)c->tiles_per_row;
-    std::vector<int32_t> count(ntiles, 0);
-    for (int32_t t = 0; t < c->v_p; ++t)
-        if (inv[t] >= 0) ++count[t / OD_SAMPLE_TILE];
-    int32_t longest = 1;
-    for (size_t i = 0; i < ntiles; ++i) longest = count[i] > longest ? count[i] : longest;
-    const int32_t width = (longest + 31) / 32 * 32;
-    std::vector<int32_t> mt(ntiles * width, -1), md(ntiles * width, 0);
-    std::fill(count.begin(), count.end(), 0);
-    for (int32_t t = 0; t < c->v_p; ++t) {
-        if (inv[t] < 0) continue;
-        const size_t i = (size_t)t / OD_SAMPLE_TILE;
-        mt[i * width + count[i]] = t;
-        md[i * width + count[i]] = inv[t];
-        ++count[i];
-    }
-    if (c->d_mapped_t) { cudaFree(c->d_mapped_t); c->d_mapped_t = nullptr; }
-    if (c->d_mapped_d) { cudaFree(c->d_mapped_d); c->d_mapped_d = nullptr; }
-    int32_t st = dev_alloc(&c->d_mapped_t, mt.size());
-    if (st == OD_OK) st = dev_alloc(&c->d_mapped_d, md.size());
-    if (st != OD_OK) return st;
-    OD_CUDA(cudaMemcpy(c->d_mapped_t, mt.data(), mt.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
-    OD_CUDA(cudaMemcpy(c->d_mapped_d, md.data(), md.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
-    c->list_width = width;
     c->have_map = true;
     return OD_OK;
 }
@@ -270,11 +254,6 @@ int32_t od_set_option(od_ctx *c, const char *name, int64_t value)
     if (!strcmp(name, "early_inputs")) { c->opt_early_inputs = value != 0; return OD_OK; }
     if (!strcmp(name, "sample_tiles_per_warp")) { c->opt_sample_tiles_per_warp = value; return OD_OK; }
     if (!strcmp(name, "pdl")) { c->opt_pdl = value != 0; return OD_OK; }
-    if (!strcmp(name, "sample_dense")) {
-        if (value > 5) return OD_ERR_INVALID_ARG;
-        c->opt_sample_dense = value;
-        return OD_OK;
-    }
     return OD_ERR_INVALID_ARG;
 }
 

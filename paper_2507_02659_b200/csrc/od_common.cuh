@@ -12,6 +12,7 @@
 #define OD_GROUP 32                 // slots of one hash-table probe group
 #define OD_SAMPLE_TILE 256          // elements of one residual-sampler tile (8 per lane of a warp)
 #define OD_SAMPLE_THREADS 256
+#define OD_SAMPLE_SMEM_MAX (200 * 1024)  // dynamic shared memory the sampler may ask for: 8 bytes per tile
 #define OD_VERIFY_SEG_MAX 64        // most segments (partials) one logit row is cut into
 #define OD_VERIFY_MAX_B 2048        // sequences per od_verify launch (longer batches go in slices)
 
@@ -23,12 +24,6 @@ struct od_ctx {
     // vocabulary map (device)
     int32_t *d_vocab_map;           // [v_q]
     int32_t *d_inv_map;             // [v_p], -1 outside the image
-    // the mapped ids sorted by target id, as one fixed-width list per tile of
-    // OD_SAMPLE_TILE target ids: entry k of tile i is at i * list_width + k,
-    // unused entries hold target id -1 (and draft id 0)
-    int32_t *d_mapped_t;            // [tiles_per_row * list_width] target id
-    int32_t *d_mapped_d;            // [tiles_per_row * list_width] its draft id
-    int32_t list_width;             // multiple of 32, >= the longest list
     bool have_map;
 
     // n-gram cache: open addressing over groups of 32 slots
@@ -62,7 +57,6 @@ struct od_ctx {
     int64_t opt_verify_grid;        // blocks of the stream kernel (0 = one per multiprocessor)
     int64_t opt_early_inputs;       // od_verify may read logits and temperatures before griddepcontrol.wait
     int64_t opt_sample_tiles_per_warp;
-    int64_t opt_sample_dense;       // pass 1 of the sampler: 0 = automatic, 1 = lists, 2..4 = inverse map, that many tiles in flight, 5 = pipelined pairs
     int64_t opt_pdl;                // launch with programmatic stream serialization
 
     // set by the entry points for the verify launch that follows: space A may be streamed early
@@ -114,6 +108,9 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              const float *temperature, const uint64_t *seed, uint64_t step,
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
                              cudaStream_t s);
+
+size_t od_sample_smem_bytes(int32_t ntiles);            // dynamic shared memory of the sampler kernel
+cudaError_t od_sample_prepare_device(size_t bytes);     // opt in to it where it exceeds the default
 
 // vocabulary shards (columns [shard_lo, shard_lo + shard_len) of the rows on this GPU)
 cudaError_t od_launch_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo,

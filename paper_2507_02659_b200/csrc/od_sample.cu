@@ -7,26 +7,27 @@
 // Inverse-CDF sampling in target-id order over tiles of 256 ids (8 consecutive
 // ids per lane of one warp, so a tile needs shuffles only, no block barrier).
 // Values are carried unnormalised: e(t) = exp2((x_t - M)*scale) = p(t)*S and
-// r'(t) = max(0, e(t) - q'(t)*S) = e(t) - min(e(t), q'(t)*S), so that
-//   sum over a tile of r' = (sum of e over the tile) - (sum over the mapped ids t
-//   of the tile of min(e(t), q'(t)*S)).
-// Only a sixth of the target ids have a draft pre-image, and the context holds them
-// sorted by target id as one fixed-width list per tile, so:
-//   pass 1  every warp takes a run of tiles of row j = n_b; per tile it sums e over
-//           the 256 ids (coalesced 128-bit loads) minus the corrections over the tile's
-//           list (a coalesced read of the list, one gathered drafter probability and
-//           one logit, already in cache, per entry) and stores the tile's value;
+// r'(t) = max(0, e(t) - q'(t)*S).
+//   pass 1  every warp takes a run of tiles of row j = n_b; per tile one coalesced
+//           128-bit load of the logits, one coalesced read of the inverse map (the
+//           draft id of each target id, -1 outside the map's image), a predicated
+//           gather of the drafter's probability for the ids that have one, r' of
+//           its eight ids (with the two ids Eq. (2) singles out) and one warp sum:
+//           the tile's value. Whole tiles go in pairs, software-pipelined: the
+//           inverse-map entries of the next pair are requested before the gathers
+//           of the current pair, so a pair costs one memory round trip;
 //   ticket  blocks never wait for each other: the block that draws the
 //           sequence's last ticket continues alone;
 //   pass 2  that block scans the tile values in parallel (total,
 //           target = u * total), finds the tile in which the running sum crosses
 //           the target, and one warp evaluates r'(t) of that single tile id by id
-//           (through the inverse map, with the two ids Eq. (2) singles out) and
-//           scans inside it. Without residual mass it draws from p_j (it then
+//           and scans inside it. Without residual mass it draws from p_j (it then
 //           redoes the tile sums with e alone).
-// Sums and scans across lanes and tiles are fp64 in a fixed order: the result is
+// A lane adds its eight values in fp32 in index order and a tile's value is the
+// fp32 warp sum of the lanes (fixed shuffle tree); sums and scans across tiles,
+// and the scan inside the chosen tile, are fp64 in a fixed order: the result is
 // reproducible, and the only difference to exact arithmetic is the fp32 rounding
-// of the individual terms.
+// of the terms and of the tile sums.
 //
 // Vocabulary shards (the rows split by columns over several GPUs) use the same
 // kernel in two further modes. A shard owns a window of whole tiles:
@@ -64,8 +65,6 @@ struct SampleArgs {
     int32_t *out_token;
     float *resid_mass;
     uint32_t *flags;
-    const int32_t *mapped_t, *mapped_d;   // mapped ids: one list of list_width entries per tile
-    int32_t list_width;
     double *tile_val;                   // [B][ntiles] sum over the tile of r'
     unsigned int *ticket;
     // vocabulary shards: this shard's tiles are [tile_lo, tile_hi); `logits` points at
@@ -75,7 +74,6 @@ struct SampleArgs {
     const double *mass_all;             // [n_shards][B][2] (residual share, share of p_j or 0)
     double *mass_out;                   // [B][2] this shard's shares
     int32_t early;                      // 1: the translation's outputs may be read before griddepcontrol.wait
-    int32_t dense;                      // pass 1: 0 = through the lists, 2..4 = inverse map, that many tiles in flight, 5 = pipelined pairs
 };
 
 // what one sequence's warps need to evaluate r(t)
@@ -207,17 +205,6 @@ __device__ __forceinline__ void tile_e_values(const SeqState &q, const SampleArg
     }
 }
 
-// one entry of a tile's list: min(e(t), q'(t)*S). The id that Eq. (2) gives the
-// n-gram's probability is left to the caller; the first sub-token of the n-gram
-// carries the reduced probability.
-template <int DTYPE>
-__device__ __forceinline__ float corr_term(const SeqState &q, int32_t t, int32_t d, float x, float qd)
-{
-    if (t < 0 || t == q.ngram_token) return 0.f;
-    if (d == q.first_draft) qd = q.prefix_val;
-    return fminf(od_ex2(fmaf(x, q.scale, -q.c)), qd * q.S);
-}
-
 __device__ __forceinline__ float warp_sum_f32(float v)
 {
 #pragma unroll
@@ -225,118 +212,9 @@ __device__ __forceinline__ float warp_sum_f32(float v)
     return v;
 }
 
-// pass 1 for a batch of n <= TB consecutive tiles by one warp: the value of a tile is
-// (sum of e over its ids) - (sum of the corrections over its list). A lane adds its
-// eight e's and subtracts the corrections of the list entries it is given (lane l
-// takes entries l, l + 32, ... of the tile's list), so ONE warp sum per tile yields
-// the tile's value. This pass is bound by instruction issue and memory latency, not
-// by bandwidth: the loads of the whole batch are issued level by level (logits and
-// list bounds, then list entries, then the gathered probabilities and logits).
-template <int DTYPE, int TB>
-__device__ __forceinline__ void warp_batch(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
-                                           int n, int lane, double *tile_val, int32_t dummy)
-{
-    uint4 raw[TB][DTYPE == OD_BF16 ? 1 : 2];
-    const int whole_n = (a.v_p / OD_SAMPLE_TILE - t_lo) < n ? (a.v_p / OD_SAMPLE_TILE - t_lo) : n;   // tiles with all 256 ids
-#pragma unroll
-    for (int i = 0; i < TB; ++i) {
-        if (i < whole_n) {
-            const uint4 *src = (const uint4 *)(q.row + ((size_t)(t_lo + i) * OD_SAMPLE_TILE + lane * EPT) *
-                                                           (DTYPE == OD_BF16 ? 2 : 4));
-            raw[i][0] = __ldg(src);
-            if (DTYPE != OD_BF16) raw[i][1] = __ldg(src + 1);
-        }
-    }
-    // the first two rounds of every tile's list (its address needs no lookup: fixed width;
-    // unused entries hold -1); wider lists finish below
-    int32_t et[TB][2], ed[TB][2];
-    const int rounds = a.list_width >> 5;
-#pragma unroll
-    for (int i = 0; i < TB; ++i) {
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            const bool ok = residual && i < n && k < rounds;
-            const size_t idx = (size_t)(t_lo + i) * a.list_width + k * 32 + lane;
-            et[i][k] = ok ? __ldg(a.mapped_t + idx) : -1;
-            ed[i][k] = ok ? __ldg(a.mapped_d + idx) : 0;
-        }
-    }
-    float ex[TB][2], eq[TB][2];
-#pragma unroll
-    for (int i = 0; i < TB; ++i) {
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            const int32_t t = et[i][k] >= 0 ? et[i][k] : dummy;   // always a valid address; the term is dropped below
-            ex[i][k] = od_load_logit<DTYPE>(q.row, t);
-            eq[i][k] = __ldg(q.q_row + ed[i][k]);
-        }
-    }
-
-    const uint64_t scale2 = f2_pack(q.scale, q.scale), nc2 = f2_pack(-q.c, -q.c);
-    float mine = 0.f;
-#pragma unroll
-    for (int i = 0; i < TB; ++i) {
-        if (i < n) {                                        // n and whole_n are the same for the whole warp
-            float sum;
-            if (i < whole_n) {
-                uint64_t acc = 0ull;
-                if (DTYPE == OD_BF16) {
-                    const uint4 v = raw[i][0];
-                    acc = f2_exp_acc(acc, od_bf16_lo(v.x), od_bf16_hi(v.x), scale2, nc2);
-                    acc = f2_exp_acc(acc, od_bf16_lo(v.y), od_bf16_hi(v.y), scale2, nc2);
-                    acc = f2_exp_acc(acc, od_bf16_lo(v.z), od_bf16_hi(v.z), scale2, nc2);
-                    acc = f2_exp_acc(acc, od_bf16_lo(v.w), od_bf16_hi(v.w), scale2, nc2);
-                } else {
-                    const uint4 v0 = raw[i][0], v1 = raw[i][DTYPE == OD_BF16 ? 0 : 1];
-                    acc = f2_exp_acc(acc, __uint_as_float(v0.x), __uint_as_float(v0.y), scale2, nc2);
-                    acc = f2_exp_acc(acc, __uint_as_float(v0.z), __uint_as_float(v0.w), scale2, nc2);
-                    acc = f2_exp_acc(acc, __uint_as_float(v1.x), __uint_as_float(v1.y), scale2, nc2);
-                    acc = f2_exp_acc(acc, __uint_as_float(v1.z), __uint_as_float(v1.w), scale2, nc2);
-                }
-                float s0, s1;
-                f2_unpack(acc, s0, s1);
-                sum = s0 + s1;
-            } else {
-                float r[EPT];
-                tile_e_values<DTYPE>(q, a, t_lo + i, lane, r);   // the ragged last tile, id by id
-                sum = r[0];
-#pragma unroll
-                for (int e = 1; e < EPT; ++e) sum += r[e];
-            }
-            if (residual) {
-#pragma unroll
-                for (int k = 0; k < 2; ++k) sum -= corr_term<DTYPE>(q, et[i][k], ed[i][k], ex[i][k], eq[i][k]);
-                for (int k = 2; k < rounds; ++k) {              // a wide list
-                    const size_t idx = (size_t)(t_lo + i) * a.list_width + k * 32 + lane;
-                    const int32_t t = __ldg(a.mapped_t + idx), d = __ldg(a.mapped_d + idx);
-                    sum -= corr_term<DTYPE>(q, t, d, od_load_logit<DTYPE>(q.row, t >= 0 ? t : dummy), __ldg(q.q_row + d));
-                }
-                // the n-gram's own token carries the n-gram's probability
-                if (lane == 0 && q.ngram_token >= 0 && q.ngram_token < a.v_p &&
-                    q.ngram_token / OD_SAMPLE_TILE == t_lo + i)
-                    sum -= fminf(od_ex2(fmaf(od_load_logit<DTYPE>(q.row, q.ngram_token), q.scale, -q.c)),
-                                 q.ngram_prob * q.S);
-            }
-            sum = warp_sum_f32(sum);
-            if (lane == i) mine = sum;
-        }
-    }
-    if (lane < n) tile_val[t_lo + lane] = (double)mine;
-}
-
-template <int DTYPE>
-__device__ __forceinline__ void warp_tiles(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
-                                           int t_hi, int lane, double *tile_val, int32_t dummy)
-{
-    constexpr int TB = 4;
-    for (int t = t_lo; t < t_hi; t += TB)
-        warp_batch<DTYPE, TB>(q, a, residual, t, t_hi - t < TB ? t_hi - t : TB, lane, tile_val, dummy);
-}
-
-// Pass 1 without the lists: every id of a tile looks up its draft id in the inverse map
-// (coalesced) and gathers the drafter's probability if it has one. Per id this moves more
-// bytes than the lists do (the inverse map is twice the size of a bf16 row, but it stays in
-// L2), and it takes far fewer instructions per tile; NT tiles are in flight per warp.
+// Pass 1, tile by tile (the free token, ragged last tiles, and the fallback of pass 2): every
+// id of a tile looks up its draft id in the inverse map (coalesced) and gathers the drafter's
+// probability if it has one; NT tiles are in flight per warp.
 template <int DTYPE, int NT>
 __device__ __forceinline__ void warp_tiles_dense(const SeqState &q, const SampleArgs &a, bool residual, int t_lo,
                                                  int t_hi, int lane, double *tile_val)
@@ -523,7 +401,6 @@ od_sample_kernel(const SampleArgs a)
     // moved back by the shard's first column, and only ids of the window are read
     const int tile_lo = MODE == 0 ? 0 : a.tile_lo;
     const int tile_hi = MODE == 0 ? a.ntiles : a.tile_hi;
-    const int32_t dummy = MODE == 0 ? 0 : tile_lo * OD_SAMPLE_TILE;   // an id that is safe to load
     SeqState q;
     q.row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)j * a.row_stride) * esz;
     if (MODE != 0) q.row -= (size_t)a.col0 * esz;
@@ -579,20 +456,15 @@ od_sample_kernel(const SampleArgs a)
             int t_hi = t_lo + a.tiles_per_warp;
             if (t_hi > tile_hi) t_hi = tile_hi;
             if (t_lo < t_hi) {
-                if (a.dense == 5) {
-                    // whole tiles pipelined; the row's ragged last tile (if it is this warp's) on its own
-                    const int whole = a.v_p / OD_SAMPLE_TILE;
-                    const int hi_w = t_hi < whole ? t_hi : whole;
-                    if (q.residual) {
-                        if (t_lo < hi_w) warp_tiles_dense_piped<DTYPE>(q, a, t_lo, hi_w, lane, tile_val);
-                        if (hi_w < t_hi) warp_tiles_dense<DTYPE, 2>(q, a, true, hi_w > t_lo ? hi_w : t_lo, t_hi, lane, tile_val);
-                    } else {
-                        warp_tiles_dense<DTYPE, 2>(q, a, false, t_lo, t_hi, lane, tile_val);
-                    }
-                } else if (a.dense == 2) warp_tiles_dense<DTYPE, 2>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
-                else if (a.dense == 3) warp_tiles_dense<DTYPE, 3>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
-                else if (a.dense == 4) warp_tiles_dense<DTYPE, 4>(q, a, q.residual, t_lo, t_hi, lane, tile_val);
-                else warp_tiles<DTYPE>(q, a, q.residual, t_lo, t_hi, lane, tile_val, dummy);
+                // whole tiles pipelined; the row's ragged last tile (if it is this warp's) on its own
+                const int whole = a.v_p / OD_SAMPLE_TILE;
+                const int hi_w = t_hi < whole ? t_hi : whole;
+                if (q.residual) {
+                    if (t_lo < hi_w) warp_tiles_dense_piped<DTYPE>(q, a, t_lo, hi_w, lane, tile_val);
+                    if (hi_w < t_hi) warp_tiles_dense<DTYPE, 2>(q, a, true, hi_w > t_lo ? hi_w : t_lo, t_hi, lane, tile_val);
+                } else {
+                    warp_tiles_dense<DTYPE, 2>(q, a, false, t_lo, t_hi, lane, tile_val);
+                }
             }
         }
         // The tile values are read by another block: the barrier orders this block's stores
@@ -626,8 +498,8 @@ od_sample_kernel(const SampleArgs a)
         double mass_e = 0.0;
         if (residual && !(mass_r > 0.0)) {
             // no residual mass here: should no shard have any, the draw is from p_j
-            for (int t_lo = tile_lo + warp * 4; t_lo < tile_hi; t_lo += WARPS * 4)
-                warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 4 < tile_hi ? t_lo + 4 : tile_hi, lane, tile_val, dummy);
+            for (int t_lo = tile_lo + warp * 2; t_lo < tile_hi; t_lo += WARPS * 2)
+                warp_tiles_dense<DTYPE, 2>(q, a, false, t_lo, t_lo + 2 < tile_hi ? t_lo + 2 : tile_hi, lane, tile_val);
             __syncthreads();
             for (int t = tile_lo + threadIdx.x; t < tile_hi; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, tile_val[t]);
             __syncthreads();
@@ -767,8 +639,8 @@ od_sample_kernel(const SampleArgs a)
         // no usable residual mass: draw from p_j instead (rare; this block redoes the row)
         residual = false;
         flags |= OD_SF_ZERO_MASS;
-        for (int t_lo = warp * 4; t_lo < ntiles; t_lo += WARPS * 4)
-            warp_tiles<DTYPE>(q, a, false, t_lo, t_lo + 4 < ntiles ? t_lo + 4 : ntiles, lane, tile_val, dummy);
+        for (int t_lo = warp * 2; t_lo < ntiles; t_lo += WARPS * 2)
+            warp_tiles_dense<DTYPE, 2>(q, a, false, t_lo, t_lo + 2 < ntiles ? t_lo + 2 : ntiles, lane, tile_val);
         __syncthreads();
         for (int t = threadIdx.x; t < ntiles; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, tile_val[t]);
         __syncthreads();
@@ -781,6 +653,25 @@ od_sample_kernel(const SampleArgs a)
 }
 
 }  // namespace
+
+// Dynamic shared memory of the kernel for rows of `ntiles` tiles: the tile values of pass 2.
+size_t od_sample_smem_bytes(int32_t ntiles) { return (size_t)ntiles * 8; }
+
+// Rows beyond 6144 tiles need more dynamic shared memory than a kernel gets by default: opt
+// in (the device must be current; allocates nothing).
+cudaError_t od_sample_prepare_device(size_t bytes)
+{
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    cudaError_t e = cudaSuccess;
+    const int n = (int)bytes;
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    return e;
+}
 
 // mode 0: od_sample_residual; 1 / 2: the two calls of a vocabulary shard
 static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, const void *logits,
@@ -822,13 +713,11 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     a.vocab_map = c->d_vocab_map; a.inv_map = c->d_inv_map;
     a.out_token = out_token; a.resid_mass = resid_mass; a.flags = flags;
     a.tile_val = c->d_tile_sums; a.ticket = c->d_samp_ticket;
-    a.mapped_t = c->d_mapped_t; a.mapped_d = c->d_mapped_d; a.list_width = c->list_width;
     a.tile_lo = tile_lo; a.tile_hi = tile_hi; a.col0 = mode == 0 ? 0 : shard_lo;
     a.n_shards = n_shards; a.shard_index = shard_index; a.mass_all = mass_all; a.mass_out = mass_out;
     // the translation kernel releases its successor before it has written anything: directly
     // after it, nothing may be read early
     a.early = c->last_was_map ? 0 : 1;
-    a.dense = c->opt_sample_dense == 1 ? 0 : (c->opt_sample_dense >= 2 ? (int32_t)c->opt_sample_dense : 5);
     c->last_was_map = false;
     if (mode != 2) {
         c->info[2] = (int64_t)blocks_x * B;
@@ -838,7 +727,7 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks_x, (unsigned)B);
     cfg.blockDim = dim3(OD_SAMPLE_THREADS);
-    cfg.dynamicSmemBytes = (size_t)ntiles * 8;
+    cfg.dynamicSmemBytes = od_sample_smem_bytes(ntiles);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
