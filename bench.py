@@ -3,14 +3,17 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..6] [--impl reference]
 
-A step is one pass of the whole hot path (od_map_proposals -> od_verify ->
-od_sample_residual) over one batch of synthetic input. The default workload is
-the batched 128256-id configuration (config 4); steps cycle through a pool of
+A step is one pass of the whole hot path (od_step: od_map_proposals -> od_verify
+-> od_sample_residual) over one batch of synthetic input. The default workload
+is the batched 128256-id configuration (config 4); steps cycle through a pool of
 distinct input buffers larger than the L2 so every step's logits come from HBM.
 The K timed steps are captured into one CUDA graph (the kernels run back to back
 as in a decode loop) and timed with CUDA events between a barrier +
-synchronize on both sides; with N > 1 every rank runs its own full batch (weak
-scaling, no data-path collective) and the time is the max over ranks.
+synchronize on both sides. The graph is then replayed for about 1.5 s, each
+replay timed the same way, and `value` comes from the median replay: the
+interval in which the clocks are sampled. With N > 1 every rank runs its own
+full batch (weak scaling, no data-path collective) and the time is the max over
+ranks; `--gpus N` without a torchrun environment starts the N ranks itself.
 
 Also reported: `roofline` for od_verify (algorithmic logit bytes / its own
 average launch duration from a graph of the same K launches, against the
@@ -77,7 +80,12 @@ class ClockSampler:
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.index = index
+        # nvidia-smi numbers the physical GPUs and ignores CUDA_VISIBLE_DEVICES: ask by UUID
+        self.index = str(index)
+        try:
+            self.index = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+        except Exception:
+            pass
         self.rows = []
         self.proc = None
 
@@ -199,9 +207,9 @@ def run_reference(a):
     from paper_2507_02659_b200 import synth
     w = synth.paper_config(a.config)
     st = synth.make_static(w)
-    # one step = a bounded sample of the workload: the first sequences of a batch
-    sel = min(w.B, 16)
-    w_s = synth.scaled(w, B=sel)
+    # one step = one full batch of the configuration
+    sel = w.B
+    w_s = w
     import oracle
     cache = oracle.Cache(st.runs, st.run_len, st.run_target)
     threads = oracle.max_threads()
@@ -224,7 +232,7 @@ def run_reference(a):
             t_total += dt
             tokens += int(s.draft_len.sum())
     value = tokens / t_total
-    sample = f"{sel} of {w.B} sequences per step, {a.steps} steps"
+    sample = f"all {w.B} sequences of a step, {a.steps} steps (cycling {len(steps)} distinct steps)"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": a.gpus,
         "steps": a.steps, "warmup": a.warmup, "ms_per_step": 1e3 * t_total / a.steps,
@@ -442,8 +450,33 @@ def run_vocab_shard(a):
     ctx.close()
 
 
+def launcher_command(gpus: int, argv, port: int):
+    """The command that starts `gpus` local ranks of this script (one per GPU) the way the
+    scaling runs are started: torch.distributed.run on one node, rendezvous on 127.0.0.1."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def maybe_relaunch(a, argv, run=subprocess.call):
+    """`--gpus N` (N > 1) outside a torchrun environment: start the N ranks and return their
+    exit status; otherwise None (this process is a rank, or the only one)."""
+    if a.gpus <= 1 or "WORLD_SIZE" in os.environ:
+        return None
+    return run(launcher_command(a.gpus, argv, free_port()))
+
+
 def main():
     a = parse()
+    rc = maybe_relaunch(a, sys.argv[1:])
+    if rc is not None:
+        sys.exit(rc)
     if a.impl == "reference":
         return run_reference(a)
     if a.distill:
@@ -510,7 +543,9 @@ def main():
 
     def full_step(step):
         i = step % P
-        k1(i, step); k2(i, step); k3(i, step)
+        s = pool[i]
+        od.od_step(ctx, s.draft_ids, s.draft_len, s.q_sel, s.q_rows, s.logits, s.temperature, s.seed, step,
+                   mp=mps[i], vo=vos[i], so=sos[i])
 
     # warm-up (also fills m for the K2-only graph)
     for step in range(a.warmup):
@@ -562,12 +597,17 @@ def main():
     if rank == 0:
         clocks.start()
         time.sleep(0.3)
-    ms_step = timed(g_step, full_step)
-    # repeats of the same K steps: more samples of the clocks under this load, and a
-    # check that the first timed region was not an outlier
-    extra, t_end = [], time.perf_counter() + 1.5
+    ms_first = timed(g_step, full_step)
+    # The same K steps again and again for about 1.5 s, each replay timed like the first: the
+    # clocks are sampled over this window, and the headline number is its median replay.
+    extra, t_end = [ms_first], time.perf_counter() + 1.5
     while time.perf_counter() < t_end and len(extra) < 400:
         extra.append(timed(g_step, full_step))
+    if world > 1:                                   # every rank must take the same number of replays
+        n_rep = torch.tensor([len(extra)], device=dev)
+        dist.all_reduce(n_rep, op=dist.ReduceOp.MIN)
+        extra = extra[:int(n_rep.item())]
+    ms_step = statistics.median(extra)
     ms_k2 = timed(g_k2, lambda step: k2(step % P, step))
     ms_k3 = timed(g_k3, lambda step: k3(step % P, step))
     ms_k1 = timed(g_k1, lambda step: k1(step % P, step))
@@ -633,8 +673,20 @@ def main():
                          f"distinct steps ({el:.1f} s of oracle time)"}
 
     if rank == 0:
-        acc = sum(int(vos[i].n_accepted.sum().item()) for i in range(P))
-        prop = sum(tokens_per_slot)
+        # what the timed steps decided (the pool slots hold the outputs of their last step)
+        acc = sum(int(vos[i].n_accepted.sum().item()) for i in steps_idx)
+        acc_draft = sum(int(vos[i].n_draft_accepted.sum().item()) for i in steps_idx)
+        prop = sum(tokens_per_slot[i] for i in steps_idx)
+        mapped = sum(int(mps[i].m.clamp(0, K).sum().item()) for i in steps_idx)
+        vflag = sum(int((vos[i].flags & od.OD_VF_BOUNDARY_MASK != 0).sum().item()) for i in steps_idx)
+        vbits = sum(int(sum(((vos[i].flags >> k) & 1).sum().item() for k in range(K))) for i in steps_idx)
+        sflag = sum(int((sos[i].flags & od.OD_SF_BOUNDARY != 0).sum().item()) for i in steps_idx)
+        bonus = sum(int((sos[i].flags & od.OD_SF_BONUS != 0).sum().item()) for i in steps_idx)
+        zero = sum(int((sos[i].flags & od.OD_SF_ZERO_MASS != 0).sum().item()) for i in steps_idx)
+        stops = sum(int((mps[i].tail_kind == od.OD_TAIL_UNMAPPED_STOP).sum().item()) for i in steps_idx)
+        hits = sum(int((mps[i].span_len[torch.arange(K, device=dev)[None, :] < mps[i].m[:, None]] >= 2).sum().item())
+                   for i in steps_idx)
+        n_seq = B * a.steps
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps,
             "warmup": a.warmup, "ms_per_step": ms_max / a.steps, "higher_is_better": True,
@@ -644,13 +696,16 @@ def main():
                        "cache_entries": w.cache_entries, "pool_buffers": P,
                        "l2_policy": f"inputs larger than L2: {P} distinct step buffers, "
                                     f"{P * logit_bytes / 2**20:.0f} MiB of logits cycled",
-                       "launch": "K steps captured in one CUDA graph" if not a.no_graph else "eager launches",
+                       "launch": ("K steps (one od_step call each) captured in one CUDA graph, replayed for 1.5 s; "
+                                  "value from the median replay") if not a.no_graph else "eager launches",
+                       "roofline_launch": "od_verify alone, K calls in one graph, option early_inputs = 1 "
+                                          "(the pool's inputs are resident before any timed launch)",
                        "parallelism": f"batch sharding x{world}, no collective"},
             "gpu_launches": 4 * a.steps,
             "kernels_ms_per_step": {"od_map_proposals": ms_k1 / a.steps, "od_verify": ms_k2 / a.steps,
                                     "od_sample_residual": ms_k3 / a.steps,
-                                    "step_repeats": len(extra),
-                                    "step_repeat_median_ms": (statistics.median(extra) / a.steps) if extra else None},
+                                    "step_replays": len(extra),
+                                    "first_replay_ms_per_step": ms_first / a.steps},
             "roofline": {"kernel": "od_verify (od_verify_stream_kernel + od_verify_decide_kernel)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                          "bytes_per_launch": k2_bytes_per_launch,
@@ -658,8 +713,15 @@ def main():
                          "frac_of_theoretical_8184": achieved / 8184.0,
                          "traffic": ncu_traffic(w0.name)},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clk,
-            "stats": {"acceptance_rate": acc / max(1, prop), "rows_per_step": rows_total / a.steps,
+            "stats": {"acceptance_rate": acc_draft / max(1, prop), "rows_per_step": rows_total / a.steps,
                       "draft_tokens_per_step": tokens_local / a.steps,
+                      "mean_accepted_length": acc / n_seq,
+                      "accepted_target_tokens_per_sec": (acc + n_seq) / (ms_max * 1e-3),
+                      "mapped_target_tokens": mapped, "cache_hits": hits, "unmapped_stops": stops,
+                      "accept_decisions": mapped, "accept_decisions_flagged": vbits,
+                      "sequences_with_a_flagged_accept_decision": vflag,
+                      "extra_tokens": n_seq, "extra_tokens_flagged": sflag, "free_tokens": bonus,
+                      "zero_residual_mass": zero,
                       "verify_grid": ctx.last_launch_info(0), "verify_span_a": ctx.last_launch_info(1),
                       "sample_grid": ctx.last_launch_info(2)},
         }

@@ -377,14 +377,20 @@ int32_t od_exit_rule(od_ctx *ctx, int32_t B, int32_t K_max, const float *head_lo
  * sums of the streaming pass: it is a fixed 1 MiB array compiled into the
  * library (OD_NOALLOC_MAX_ROWS rows x 64 partials x 16 bytes) that every GPU
  * loading the library holds until the process ends. The function calls no
- * cudaMalloc, cudaFree or other allocating routine.
+ * cudaMalloc, cudaFree or other allocating routine. It always waits for the
+ * launch in front of it before it reads the logits (there is no context to
+ * carry the "early_inputs" promise), so any producer is safe.
  *
  * Limits and rules
  *   - B * (K_max + 1) <= OD_NOALLOC_MAX_ROWS and B <= 2048; anything larger is
  *     refused with OD_ERR_SCRATCH_LIMIT before any launch.
  *   - The first call on a device looks up the array's device address and the
- *     multiprocessor count (no allocation, but host-side runtime calls): make
- *     that first call during start-up, before any stream capture begins.
+ *     multiprocessor count (no allocation by this library, but host-side
+ *     runtime calls). Where the CUDA runtime loads modules lazily, that first
+ *     call is also the moment at which the driver loads the module and sets
+ *     the array's 1 MiB aside, so free device memory can drop then, once.
+ *     Make that first call during start-up, before any stream capture begins
+ *     and before memory is tight.
  *   - All calls on a device share the one array. It keeps whatever the last
  *     call left in it; nothing in it needs clearing, because a call reads only
  *     the slots it has written itself. Two calls whose kernels overlap on the

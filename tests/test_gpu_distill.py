@@ -87,3 +87,33 @@ def test_random_shapes(cuda_device, i):
                logit_dtype=["bf16", "f32"][int(rng.integers(0, 2))], mapped_frac=float(rng.uniform(0.3, 0.9)),
                cache_entries=int(rng.integers(0, 200)), gen_seed=0xBEEFE0 + i)
     _check(w, cuda_device, range(2), lam=float(rng.uniform(0.05, 1.0)), mode=int(rng.integers(0, 2)))
+
+
+@pytest.mark.parametrize("v_q", [600, 333])
+def test_loss_without_a_gradient_buffer(cuda_device, v_q):
+    """grad = NULL: the kernel has nowhere to park q*g between its sweeps and recomputes it; the
+    loss must be the oracle's all the same (vector path for V_q = 600, scalar path for 333)."""
+    w = _small(B=10, v_q=v_q, v_p=1003, cache_entries=150, gen_seed=0xBEEFD7)
+    st = synth.make_static(w)
+    ctx = parity.make_context(w, st, cuda_device)
+    for step in range(3):
+        s = synth.make_step(w, st, step, device=cuda_device)
+        logits = parity.pad_rows(s.logits)
+        mp = od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel)
+        vo = od.od_verify(ctx, logits, mp, s.temperature, s.seed, step)
+        loss, grad = od.od_distill_loss(ctx, s.q_rows, s.draft_ids, mp, logits, vo, s.temperature, 0.2,
+                                        ds.LAMBDA_CONSTANT, want_grad=False)
+        with_grad, _ = od.od_distill_loss(ctx, s.q_rows, s.draft_ids, mp, logits, vo, s.temperature, 0.2,
+                                          ds.LAMBDA_CONSTANT)
+        torch.cuda.synchronize()
+        assert grad is None
+        m = mp.m.cpu().numpy(); ss = mp.span_start.cpu().numpy(); sl = mp.span_len.cpu().numpy()
+        tg = mp.tgt_ids.cpu().numpy(); d = s.draft_ids.cpu().numpy(); T = s.temperature.cpu().numpy()
+        loss = loss.cpu().numpy()
+        for b in range(w.B):
+            want_l, _ = ds.distill_sequence(s.q_rows[b].cpu().numpy().astype(np.float64), d[b], ss[b], sl[b], m[b],
+                                            _logits64(s.logits[b]), float(T[b]), st.vocab_map, tg[b], 0.2,
+                                            ds.LAMBDA_CONSTANT)
+            np.testing.assert_allclose(loss[b], want_l, rtol=2e-5, atol=2e-6)
+        np.testing.assert_allclose(loss, with_grad.cpu().numpy(), rtol=1e-6, atol=1e-7)
+    ctx.close()

@@ -235,6 +235,74 @@ def test_sampling_directly_after_the_translation_gives_the_same_token(cuda_devic
     ctx.close()
 
 
+def test_a_producer_directly_in_front_of_the_step_is_safe(cuda_device):
+    """The logits are written by the launch directly in front of the library's first kernel (as a
+    target model's output layer would), over rows that held NaN until then. With the default
+    options nothing may be read before that launch has finished: od_step (whose streaming kernel
+    starts on rows 0 early, behind its own translation kernel), od_verify on its own, and
+    od_verify_noalloc must all match the oracle, every time."""
+    w = _small("producer", B=48, v_q=3000, v_p=40000, cache_entries=1000, gen_seed=0xBEEF66)
+    st = synth.make_static(w)
+    ctx = parity.make_context(w, st, cuda_device)
+    cache = oracle.Cache(st.runs, st.run_len, st.run_target)
+    s = synth.make_step(w, st, 0, device=cuda_device)
+    clean = s.logits.clone()
+    temps = s.temperature.clone()
+    ref = None
+    for rep in range(20):
+        which = rep % 3
+        mp = od.alloc_map_out(ctx, w.B, w.k_max)
+        if which != 0:
+            od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel, out=mp)
+        vo = od.alloc_verify_out(ctx, w.B, w.k_max)
+        so = od.alloc_sample_out(ctx, w.B)
+        s.logits.fill_(float("nan"))
+        s.temperature.fill_(float("nan"))
+        torch.cuda.synchronize()
+        s.temperature.copy_(temps)
+        s.logits.copy_(clean)                       # the producer: the launch directly in front
+        if which == 0:
+            od.od_step(ctx, s.draft_ids, s.draft_len, s.q_sel, s.q_rows, s.logits, s.temperature, s.seed, s.step,
+                       mp=mp, vo=vo, so=so)
+        else:
+            if which == 1:
+                od.od_verify(ctx, s.logits, mp, s.temperature, s.seed, s.step, out=vo)
+            else:
+                od.od_verify_noalloc(w.v_p, s.logits, mp, s.temperature, s.seed, s.step, out=vo)
+            od.od_sample_residual(ctx, s.logits, vo, s.q_rows, s.draft_ids, mp, s.temperature, s.seed, s.step, out=so)
+        torch.cuda.synchronize()
+        if ref is None:
+            ref = parity.oracle_step(cache, st, w, s.to("cpu"), probe=so.out_token.cpu().numpy())
+            first = [t.clone() for t in (vo.row_sum, vo.n_accepted, so.out_token)]
+        parity.compare(mp, vo, so, ref, s.draft_len.cpu().numpy(), s.step,
+                       s.seed.cpu().numpy().astype(np.uint64), bf16=True)
+        assert torch.equal(vo.n_accepted, first[1]) and torch.equal(so.out_token, first[2])
+    ctx.close()
+
+
+def test_od_step_equals_the_three_calls(cuda_device):
+    w = _small("onecall", B=40, v_q=3000, v_p=30011, cache_entries=800, gen_seed=0xBEEF67)
+    st = synth.make_static(w)
+    ctx = parity.make_context(w, st, cuda_device)
+    s = synth.make_step(w, st, 3, device=cuda_device)
+    lg = parity.pad_rows(s.logits)
+    mp, vo, so = parity.gpu_step(ctx, s, logits=lg)
+    mp2, vo2, so2 = od.od_step(ctx, s.draft_ids, s.draft_len, s.q_sel, s.q_rows, lg, s.temperature, s.seed, s.step)
+    torch.cuda.synchronize()
+    m = mp.m.clamp(0, w.k_max)
+    rows = torch.arange(w.k_max + 1, device=cuda_device)[None, :] <= m[:, None]
+    pos = torch.arange(w.k_max, device=cuda_device)[None, :] < m[:, None]
+    assert torch.equal(mp.m, mp2.m) and torch.equal(mp.tgt_ids[pos], mp2.tgt_ids[pos])
+    assert torch.equal(mp.tail_kind, mp2.tail_kind) and torch.equal(mp.counters, mp2.counters)
+    assert torch.equal(vo.row_sum[rows], vo2.row_sum[rows]) and torch.equal(vo.row_max[rows], vo2.row_max[rows])
+    assert torch.equal(vo.p_sel[pos], vo2.p_sel[pos]) and torch.equal(vo.ratio[pos], vo2.ratio[pos])
+    assert torch.equal(vo.n_accepted, vo2.n_accepted) and torch.equal(vo.n_draft_accepted, vo2.n_draft_accepted)
+    assert torch.equal(vo.flags, vo2.flags)
+    assert torch.equal(so.out_token, so2.out_token) and torch.equal(so.flags, so2.flags)
+    assert torch.equal(so.resid_mass, so2.resid_mass)
+    ctx.close()
+
+
 def test_rows_above_m_are_never_read(cuda_device):
     """Rows m_b+1.. hold NaN: any touch would poison the sums."""
     w = _small("nan", B=32, gen_seed=0xBEEF70)
@@ -402,6 +470,9 @@ def test_argument_validation(cuda_device):
         big_ctx.cache_build(np.array([[1, 2, -1, -1]], np.int32), np.array([2], np.int32), np.array([7], np.int32))
     assert e.value.status == -5
     big_ctx.close()
+    with pytest.raises(od.OdError) as e:                    # the sampler could not hold a row's tile values
+        od.Context(cuda_device, 100, 7_000_000, 1, 2)
+    assert e.value.status == -5
     torch.cuda.synchronize()
     ctx.close()
 
