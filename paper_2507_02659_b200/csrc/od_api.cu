@@ -351,6 +351,21 @@ int32_t od_step(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids, c
     // kernel start, so whatever wrote the logits has finished by the time a block of the
     // stream kernel runs: rows 0 may be read before that kernel's own wait.
     c->verify_early = true;
+    if (B > 0 && B <= od_verify_slice(K_max, c->v_p, logit_dtype) && c->opt_pdl) {
+        // Three launches, not four: the streaming pass, then the sampler, whose blocks merge the
+        // pass's partials and take step 2's decisions themselves (identical arithmetic) instead
+        // of waiting for a decide kernel in between.
+        od_fused_verify fuse = {};
+        fuse.row_max = row_max; fuse.row_sum = row_sum; fuse.p_sel = p_sel; fuse.ratio = ratio;
+        fuse.n_accepted = n_accepted; fuse.n_draft_accepted = n_draft_accepted; fuse.flags = verify_flags;
+        OD_CUDA(od_launch_verify_stream(c, B, K_max, logits, logit_dtype, row_stride, seq_stride, m, temperature,
+                                        &fuse, s));
+        OD_CUDA(od_launch_sample(c, B, K_max, logits, logit_dtype, row_stride, seq_stride, row_max, row_sum,
+                                 q_rows, draft_ids, tgt_ids, q_prime, span_start, span_len, m, tail_kind,
+                                 n_accepted, temperature, seed, step, out_token, resid_mass, sample_flags, s,
+                                 &fuse));
+        return OD_OK;
+    }
     OD_CUDA(od_launch_verify(c, B, K_max, logits, logit_dtype, row_stride, seq_stride, tgt_ids, q_prime,
                              span_len, m, temperature, seed, step, row_max, row_sum, p_sel, ratio,
                              n_accepted, n_draft_accepted, verify_flags, s));

@@ -98,6 +98,19 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              uint32_t *flags, cudaStream_t s);
 
 
+// od_step: the streaming pass of step 2 alone (no decide kernel), and what the sampler then needs
+// to take step 2's decisions itself: the split of the pass and where step 2's outputs go.
+struct od_fused_verify {
+    int32_t W, n_chunks, span_min, span_a;
+    float *row_max, *row_sum, *p_sel, *ratio;
+    int32_t *n_accepted, *n_draft_accepted;
+    uint32_t *flags;
+};
+int32_t od_verify_slice(int32_t K_max, int32_t v_len, int32_t dtype);   // sequences one stream launch takes
+cudaError_t od_launch_verify_stream(od_ctx *c, int32_t B, int32_t K_max, const void *logits, int32_t dtype,
+                                    int64_t row_stride, int64_t seq_stride, const int32_t *m,
+                                    const float *temperature, od_fused_verify *plan, cudaStream_t s);
+
 cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
                              int32_t dtype, int64_t row_stride, int64_t seq_stride,
                              const float *row_max, const float *row_sum, const float *q_rows,
@@ -107,7 +120,7 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              const uint8_t *tail_kind, const int32_t *n_accepted,
                              const float *temperature, const uint64_t *seed, uint64_t step,
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
-                             cudaStream_t s);
+                             cudaStream_t s, const od_fused_verify *fuse = nullptr);
 
 size_t od_sample_smem_bytes(int32_t ntiles);            // dynamic shared memory of the sampler kernel
 cudaError_t od_sample_prepare_device(size_t bytes);     // opt in to it where it exceeds the default

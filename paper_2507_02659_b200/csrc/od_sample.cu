@@ -41,6 +41,7 @@
 #include <float.h>
 
 #include "od_common.cuh"
+#include "od_decide.cuh"
 
 namespace {
 
@@ -74,6 +75,13 @@ struct SampleArgs {
     const double *mass_all;             // [n_shards][B][2] (residual share, share of p_j or 0)
     double *mass_out;                   // [B][2] this shard's shares
     int32_t early;                      // 1: the translation's outputs may be read before griddepcontrol.wait
+    // od_step: no decide kernel ran; the decisions of step 2 are taken here, by every block of a
+    // sequence alike, from the partials the streaming pass left, and the sequence's block 0
+    // writes step 2's outputs (the w_ pointers; row_max, row_sum, n_accepted above are not read)
+    StreamPlan plan;
+    float *w_row_max, *w_row_sum, *w_p_sel, *w_ratio;
+    int32_t *w_n_accepted, *w_n_draft;
+    uint32_t *w_vflags;
 };
 
 // what one sequence's warps need to evaluate r(t)
@@ -334,10 +342,16 @@ __device__ __forceinline__ double block_total(const double *s_val, int my_lo, in
 }
 
 // MODE 0: the whole step on full rows; 1: a shard's mass shares; 2: a shard's pick.
-template <int DTYPE, int MODE>
+// FUSED (mode 0 only): the launch in front is the streaming pass of od_verify itself; its
+// decide kernel is folded into this kernel's prologue (see SampleArgs).
+template <int DTYPE, int MODE, bool FUSED>
 __global__ void __launch_bounds__(OD_SAMPLE_THREADS, 4)
 od_sample_kernel(const SampleArgs a)
 {
+    __shared__ float s_M[FUSED ? OD_MAX_K + 1 : 1], s_S[FUSED ? OD_MAX_K + 1 : 1];
+    __shared__ int s_red[2][WARPS];
+    __shared__ int s_n;
+    __shared__ unsigned int s_vbits;
     extern __shared__ __align__(16) unsigned char s_dyn[];   // ntiles x 8 bytes
     double *s_val = (double *)s_dyn;                         // pass 2: tile values
     __shared__ double s_warp[WARPS];
@@ -379,8 +393,83 @@ od_sample_kernel(const SampleArgs a)
         }
     }
 
+    // FUSED, still before the wait: where the rows' partials will be (sums of m), and position
+    // k's inputs of the acceptance test in lane k
+    int before = 0, total = 0;
+    float d_xt = 0.f, d_q = 0.f, d_u = 0.f;
+    bool d_tok = false;
+    int32_t d_span = 0;
+    if (FUSED) {
+        for (int i = threadIdx.x; i < a.B; i += OD_SAMPLE_THREADS) {
+            const int v = clamp_m(a.m[i], K);
+            total += v;
+            if (i < b) before += v;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            before += __shfl_xor_sync(0xFFFFFFFFu, before, off);
+            total += __shfl_xor_sync(0xFFFFFFFFu, total, off);
+        }
+        if (lane == 0) { s_red[0][warp] = before; s_red[1][warp] = total; }
+        if (threadIdx.x == 0) s_vbits = 0;
+        if (lane < mb) {
+            const size_t o = (size_t)b * K + lane;
+            const int32_t t = a.tgt_ids[o];
+            d_tok = t >= 0 && t < a.v_p;
+            const char *row_k = (const char *)a.logits +
+                                ((size_t)b * a.seq_stride + (size_t)lane * a.row_stride) * (DTYPE == OD_BF16 ? 2 : 4);
+            if (d_tok) d_xt = od_load_logit<DTYPE>(row_k, t);
+            d_q = a.q_prime[o];
+            d_u = od_uniform(a.seed[b], a.step, (uint32_t)lane, 0u);
+            d_span = a.span_len[o];
+        }
+        __syncthreads();
+        before = 0; total = 0;
+        for (int w = 0; w < WARPS; ++w) { before += s_red[0][w]; total += s_red[1][w]; }
+    }
+
     // n_accepted and the row statistics come from the verification kernels
     if (a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    if (FUSED) {
+        // ---- step 2's decisions (what od_verify_decide_kernel does, same arithmetic, same order)
+        const bool bad_T = !(T > 0.f);
+        const float dscale = bad_T ? 0.f : 1.4426950408889634f / T;
+        for (int r = warp; r <= mb; r += WARPS) {
+            const int row_slot = b * (K + 1) + r;
+            float c, sum, mx;
+            merge_row_partials(a.plan, row_slot, row_partial_segments(a.plan, b, r, before, total), lane, c, sum, mx);
+            if (lane == 0) {
+                const float S = row_sum_of(c, sum, mx, dscale);
+                s_M[r] = mx; s_S[r] = S;
+                if (blockIdx.x == 0) { a.w_row_max[row_slot] = mx; a.w_row_sum[row_slot] = S; }
+                if (!(S > 0.f) || !(S <= FLT_MAX)) atomicOr(&s_vbits, 1u);
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            bool acc = false, bnd = false;
+            if (lane < mb) {
+                const Acceptance d = accept_position(s_M[lane], s_S[lane], dscale, d_tok, d_xt, d_q, d_u);
+                acc = d.accept; bnd = d.boundary;
+                if (blockIdx.x == 0) { a.w_p_sel[(size_t)b * K + lane] = d.p; a.w_ratio[(size_t)b * K + lane] = d.ratio; }
+            }
+            const unsigned int accmask = __ballot_sync(0xFFFFFFFFu, acc), bndmask = __ballot_sync(0xFFFFFFFFu, bnd);
+            int n = 0;
+            while (n < mb && (accmask >> n & 1u)) ++n;
+            int nd = lane < n ? d_span : 0;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) nd += __shfl_xor_sync(0xFFFFFFFFu, nd, off);
+            if (lane == 0) {
+                uint32_t f = bndmask & OD_VF_BOUNDARY_MASK;
+                if (s_vbits & 1u) f |= OD_VF_NONFINITE;
+                if (bad_T) { f |= OD_VF_BAD_TEMPERATURE; n = 0; nd = 0; }
+                s_n = n;
+                if (blockIdx.x == 0) { a.w_n_accepted[b] = n; a.w_n_draft[b] = nd; a.w_vflags[b] = f; }
+            }
+        }
+        __syncthreads();
+    }
 
     if (!(T > 0.f)) {                              // every block of the sequence leaves here
         if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -393,8 +482,11 @@ od_sample_kernel(const SampleArgs a)
         return;
     }
     float rm = 0.f, rs = 0.f;                      // lane k: statistics of row k
-    if (lane <= mb) { rm = a.row_max[b * (K + 1) + lane]; rs = a.row_sum[b * (K + 1) + lane]; }
-    int j = a.n_accepted[b];
+    if (lane <= mb) {
+        rm = FUSED ? s_M[lane] : a.row_max[b * (K + 1) + lane];
+        rs = FUSED ? s_S[lane] : a.row_sum[b * (K + 1) + lane];
+    }
+    int j = FUSED ? s_n : a.n_accepted[b];
     j = j < 0 ? 0 : (j > mb ? mb : j);
     const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
     // a shard's tiles and ids keep their numbers of the full row: the row pointer is
@@ -664,12 +756,14 @@ cudaError_t od_sample_prepare_device(size_t bytes)
     if (bytes <= 48 * 1024) return cudaSuccess;
     cudaError_t e = cudaSuccess;
     const int n = (int)bytes;
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_BF16, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(od_sample_kernel<OD_F32, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
     return e;
 }
 
@@ -684,7 +778,8 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
                                  const float *temperature, const uint64_t *seed, uint64_t step,
                                  int32_t *out_token, float *resid_mass, uint32_t *flags,
                                  int32_t shard_lo, int32_t shard_len, int32_t n_shards, int32_t shard_index,
-                                 const double *mass_all, double *mass_out, cudaStream_t s)
+                                 const double *mass_all, double *mass_out, cudaStream_t s,
+                                 const od_fused_verify *fuse = nullptr)
 {
     if (B == 0) return cudaSuccess;
     const int ntiles = c->tiles_per_row;
@@ -718,6 +813,12 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     // the translation kernel releases its successor before it has written anything: directly
     // after it, nothing may be read early
     a.early = c->last_was_map ? 0 : 1;
+    if (fuse) {
+        a.plan.W = fuse->W; a.plan.n_chunks = fuse->n_chunks; a.plan.span_min = fuse->span_min;
+        a.plan.span_a = fuse->span_a; a.plan.partials = c->d_partials;
+        a.w_row_max = fuse->row_max; a.w_row_sum = fuse->row_sum; a.w_p_sel = fuse->p_sel; a.w_ratio = fuse->ratio;
+        a.w_n_accepted = fuse->n_accepted; a.w_n_draft = fuse->n_draft_accepted; a.w_vflags = fuse->flags;
+    }
     c->last_was_map = false;
     if (mode != 2) {
         c->info[2] = (int64_t)blocks_x * B;
@@ -735,14 +836,17 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     cfg.attrs = attr;
     cfg.numAttrs = c->opt_pdl ? 1 : 0;
     const bool bf = dtype == OD_BF16;
+    if (mode == 0 && fuse)
+        return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 0, true>, a)
+                  : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 0, true>, a);
     if (mode == 0)
-        return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 0>, a)
-                  : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 0>, a);
+        return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 0, false>, a)
+                  : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 0, false>, a);
     if (mode == 1)
-        return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 1>, a)
-                  : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 1>, a);
-    return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 2>, a)
-              : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 2>, a);
+        return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 1, false>, a)
+                  : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 1, false>, a);
+    return bf ? cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_BF16, 2, false>, a)
+              : cudaLaunchKernelEx(&cfg, od_sample_kernel<OD_F32, 2, false>, a);
 }
 
 cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
@@ -754,11 +858,12 @@ cudaError_t od_launch_sample(od_ctx *c, int32_t B, int32_t K_max, const void *lo
                              const uint8_t *tail_kind, const int32_t *n_accepted,
                              const float *temperature, const uint64_t *seed, uint64_t step,
                              int32_t *out_token, float *resid_mass, uint32_t *flags,
-                             cudaStream_t s)
+                             cudaStream_t s, const od_fused_verify *fuse)
 {
     return launch_sample(c, 0, B, K_max, logits, dtype, row_stride, seq_stride, row_max, row_sum, q_rows,
                          draft_ids, tgt_ids, q_prime, span_start, span_len, m, tail_kind, n_accepted,
-                         temperature, seed, step, out_token, resid_mass, flags, 0, 0, 1, 0, nullptr, nullptr, s);
+                         temperature, seed, step, out_token, resid_mass, flags, 0, 0, 1, 0, nullptr, nullptr, s,
+                         fuse);
 }
 
 cudaError_t od_launch_sample_shard_mass(od_ctx *c, int32_t B, int32_t K_max, int32_t shard_lo,

@@ -47,11 +47,13 @@
 #include <float.h>
 
 #include "od_common.cuh"
+#include "od_decide.cuh"
 
 namespace {
 
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
+static_assert(WARPS == OD_STREAM_WARPS, "partials per block segment");
 constexpr int U = 4;                            // 16-byte loads in flight per thread
 constexpr int A_PARK = 8;                       // partials of space A a block can hold back
 #ifndef OD_VERIFY_MAXNREG
@@ -89,21 +91,6 @@ struct VerifyArgs {
     const float4 *stats_all;            // [n_shards][rows][4], rows = batch * (K_max + 1)
     int64_t stats_rows;
 };
-
-// How many blocks hold pieces of flat row `rho` of a space whose blocks take
-// `span` units each.
-__device__ __forceinline__ int row_segments(uint32_t rho, uint32_t W, uint32_t span)
-{
-    return (int)(((rho + 1) * W - 1) / span - rho * W / span + 1);
-}
-
-__device__ __forceinline__ uint32_t span_of_space_b(uint32_t rows_b, uint32_t W, uint32_t n_chunks, uint32_t span_min)
-{
-    const uint32_t span = (rows_b * W + n_chunks - 1) / n_chunks;
-    return span < span_min ? span_min : span;
-}
-
-__device__ __forceinline__ int clamp_m(int mb, int K_max) { return mb < 0 ? 0 : (mb > K_max ? K_max : mb); }
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
 {
@@ -198,29 +185,6 @@ __device__ __forceinline__ void absorb_one(Lane<DTYPE> &L, float x, float scale)
     }
     L.raise(x, scale);
     L.s += od_ex2(fmaf(x, scale, -L.c));
-}
-
-// (c, s) pairs: s counts exp2(x*scale - c)
-__device__ __forceinline__ void pair_merge(float &c, float &s, float c2, float s2)
-{
-    const float cm = fmaxf(c, c2);
-    s = s * od_ex2(c - cm) + s2 * od_ex2(c2 - cm);
-    c = cm;
-}
-
-// all lanes end with the merged (c, s, mx): one rescale per lane, then plain reductions
-__device__ __forceinline__ void warp_merge(float &c, float &s, float &mx)
-{
-    float cm = c;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        cm = fmaxf(cm, __shfl_xor_sync(0xFFFFFFFFu, cm, off));
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-    }
-    s *= od_ex2(c - cm);
-    c = cm;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
 }
 
 // Units [v0, v1) of row (b, r) by the whole block; warp w stores its partial to dst[w]
@@ -443,19 +407,18 @@ __device__ __forceinline__ void decide_row(const VerifyArgs &a, int b, int r, in
 {
     const int row_slot = b * (a.K_max + 1) + r;
     const float M = mx;
-    const float S = s * od_ex2(fmaf(-M, scale, c));     // sum of exp2((x - M)*scale)
+    const float S = row_sum_of(c, s, mx, scale);        // sum of exp2((x - M)*scale)
     a.row_max[row_slot] = M;
     a.row_sum[row_slot] = S;
     if (!(S > 0.f) || !(S <= FLT_MAX)) atomicOr(&s_bits[1], 1u);   // not finite and positive
     if (r < mb) {
         const size_t o = (size_t)b * a.K_max + r;
-        const float p = t_ok ? od_ex2((x_t - M) * scale) / S : 0.f;
-        const float ra = (q <= p) ? 1.f : p / q;
-        a.p_sel[o] = p;
-        a.ratio[o] = ra;
+        const Acceptance d = accept_position(M, S, scale, t_ok, x_t, q, u);
+        a.p_sel[o] = d.p;
+        a.ratio[o] = d.ratio;
         unsigned int bits = 0;
-        if (u < ra) bits |= 1u << r;
-        if (fabsf(u - ra) <= OD_TAU_ACCEPT) bits |= 1u << (16 + r);
+        if (d.accept) bits |= 1u << r;
+        if (d.boundary) bits |= 1u << (16 + r);
         if (bits) atomicOr(&s_bits[0], bits);
     }
 }
@@ -552,14 +515,10 @@ od_verify_decide_kernel(const VerifyArgs a)
 
     if (r <= mb) {
         const int row_slot = b * (a.K_max + 1) + r;
-        const float4 *pp = a.partials + (size_t)row_slot * OD_VERIFY_SEG_MAX;
-        float c = -FLT_MAX, s = 0.f, mx = -INFINITY;
-        for (int k = lane; k < nseg * WARPS; k += 32) {
-            const float4 p = __ldcg(pp + k);
-            pair_merge(c, s, p.x, p.y);
-            mx = fmaxf(mx, p.z);
-        }
-        warp_merge(c, s, mx);
+        StreamPlan plan;
+        plan.partials = a.partials;
+        float c, s, mx;
+        merge_row_partials(plan, row_slot, nseg, lane, c, s, mx);
         if (SHARD) {
             if (lane == 0) a.stats[row_slot] = make_float4(c, s, mx, t_ok ? x_t : -INFINITY);
         } else {
@@ -666,6 +625,28 @@ static int32_t slice_of(int32_t K_max, int32_t v_len, int32_t dtype)
     int32_t slice = OD_VERIFY_MAX_B;
     while (slice > 1 && (int64_t)slice * (K_max + 1) * W > (int64_t)1 << 30) slice >>= 1;
     return slice;
+}
+
+int32_t od_verify_slice(int32_t K_max, int32_t v_len, int32_t dtype) { return slice_of(K_max, v_len, dtype); }
+
+// The streaming pass alone, for a batch that fits one launch (B <= od_verify_slice): the
+// caller's next kernel merges the partials itself (od_step).
+cudaError_t od_launch_verify_stream(od_ctx *c, int32_t B, int32_t K_max, const void *logits, int32_t dtype,
+                                    int64_t row_stride, int64_t seq_stride, const int32_t *m,
+                                    const float *temperature, od_fused_verify *plan, cudaStream_t s)
+{
+    c->last_was_map = false;
+    VerifyArgs a = {};
+    plan_stream(c, B, K_max, c->v_p, dtype, c->verify_early, a);
+    a.logits = logits; a.row_stride = row_stride; a.seq_stride = seq_stride;
+    a.m = m; a.temperature = temperature;
+    a.partials = c->d_partials;
+    c->info[0] = a.n_chunks;
+    c->info[1] = a.span_a;
+    plan->W = a.W; plan->n_chunks = a.n_chunks; plan->span_min = a.span_min; plan->span_a = a.span_a;
+    const bool pdl = c->opt_pdl != 0;
+    return dtype == OD_BF16 ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)a.n_chunks, THREADS, s, pdl, a)
+                            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)a.n_chunks, THREADS, s, pdl, a);
 }
 
 cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
