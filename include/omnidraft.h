@@ -182,7 +182,11 @@ int32_t od_cache_set_clock(od_ctx *ctx, uint32_t clock);
  * if they were added one after the other; malformed candidates (length, ids or
  * target out of range) are skipped. New entries get the current clock as time of
  * insertion and of last access, and frequency 1. Asynchronous on `stream`; must be
- * ordered with od_map_proposals on the same context. N <= max_insert. */
+ * ordered with od_map_proposals on the same context. N <= max_insert.
+ * The table is sized for max_entries + max_insert entries at load 1/2: trim at
+ * least once per batch that can take the cache past max_entries. A candidate that
+ * finds no free slot on its whole probe sequence (only possible when trims were
+ * skipped for many batches) is dropped without a trace. */
 int32_t od_cache_insert(od_ctx *ctx, int32_t N, const int32_t *runs,
                         const int32_t *len, const int32_t *target, void *stream);
 
@@ -190,7 +194,11 @@ int32_t od_cache_insert(od_ctx *ctx, int32_t N, const int32_t *runs,
  * come first in the order (inserted at the current clock? no before yes; then last
  * access clock for LRU or frequency for LFU, ascending; then the run's packed key,
  * ascending) and rebuilds the table. Asynchronous on `stream` (a fixed sequence of
- * small kernels, no host round trip); calls enqueued afterwards see the new table. */
+ * small kernels, no host round trip); calls enqueued afterwards see the new table.
+ * The table's address and the clock are arguments of the kernels that use them: a
+ * CUDA graph that captured od_map_proposals (or od_step) keeps the table and the
+ * clock of its capture and must be captured again after od_cache_trim or
+ * od_cache_set_clock. */
 int32_t od_cache_trim(od_ctx *ctx, void *stream);
 
 /* Contents of the online cache, for inspection and tests: synchronises the device,
