@@ -251,21 +251,27 @@ __device__ __forceinline__ void warp_tiles_dense(const SeqState &q, const Sample
     }
 }
 
-// The same pass for a residual draw, software-pipelined over pairs of WHOLE tiles: the
-// inverse-map entries of the next pair are requested before the current pair's gathers,
-// so a pair costs one memory round trip, not two.
-template <int DTYPE>
-__device__ __forceinline__ void warp_tiles_dense_piped(const SeqState &q, const SampleArgs &a, int t_lo, int t_hi,
-                                                       int lane, double *tile_val)
+// Inverse-map entries of a warp's first pair of whole tiles [t_lo, t_hi).
+__device__ __forceinline__ void first_pair_entries(const SampleArgs &a, int t_lo, int t_hi, int lane, int4 (&ni)[2][2])
 {
-    constexpr int ESZ = DTYPE == OD_BF16 ? 2 : 4;
-    int4 ni[2][2];
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int t0 = (t_lo + i < t_hi ? t_lo + i : t_lo) * OD_SAMPLE_TILE + lane * EPT;
         ni[i][0] = __ldg((const int4 *)(a.inv_map + t0));
         ni[i][1] = __ldg((const int4 *)(a.inv_map + t0) + 1);
     }
+}
+
+// The same pass for a residual draw, software-pipelined over pairs of WHOLE tiles: the
+// inverse-map entries of the next pair are requested before the current pair's gathers,
+// so a pair costs one memory round trip, not two. ni: the first pair's entries
+// (first_pair_entries), which the caller requested early: they belong to the context and
+// depend on nothing the launch in front writes.
+template <int DTYPE>
+__device__ __forceinline__ void warp_tiles_dense_piped(const SeqState &q, const SampleArgs &a, int t_lo, int t_hi,
+                                                       int lane, double *tile_val, int4 (&ni)[2][2])
+{
+    constexpr int ESZ = DTYPE == OD_BF16 ? 2 : 4;
     for (int t = t_lo; t < t_hi; t += 2) {
         int32_t d[2][EPT];
 #pragma unroll
@@ -428,6 +434,17 @@ od_sample_kernel(const SampleArgs a)
         for (int w = 0; w < WARPS; ++w) { before += s_red[0][w]; total += s_red[1][w]; }
     }
 
+    // a shard's tiles and ids keep their numbers of the full row
+    const int tile_lo = MODE == 0 ? 0 : a.tile_lo;
+    const int tile_hi = MODE == 0 ? a.ntiles : a.tile_hi;
+    // pass 1's whole tiles of this warp, and the inverse-map entries of their first pair
+    const int p_lo = tile_lo + (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
+    int p_hi = p_lo + a.tiles_per_warp;
+    if (p_hi > tile_hi) p_hi = tile_hi;
+    const int p_hi_w = p_hi < a.v_p / OD_SAMPLE_TILE ? p_hi : a.v_p / OD_SAMPLE_TILE;
+    int4 ni[2][2] = {};
+    if (MODE != 2 && p_lo < p_hi_w) first_pair_entries(a, p_lo, p_hi_w, lane, ni);
+
     // n_accepted and the row statistics come from the verification kernels
     if (a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -489,10 +506,8 @@ od_sample_kernel(const SampleArgs a)
     int j = FUSED ? s_n : a.n_accepted[b];
     j = j < 0 ? 0 : (j > mb ? mb : j);
     const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
-    // a shard's tiles and ids keep their numbers of the full row: the row pointer is
-    // moved back by the shard's first column, and only ids of the window are read
-    const int tile_lo = MODE == 0 ? 0 : a.tile_lo;
-    const int tile_hi = MODE == 0 ? a.ntiles : a.tile_hi;
+    // a shard's row pointer is moved back by the shard's first column, and only ids of
+    // the window are read
     SeqState q;
     q.row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)j * a.row_stride) * esz;
     if (MODE != 0) q.row -= (size_t)a.col0 * esz;
@@ -544,15 +559,12 @@ od_sample_kernel(const SampleArgs a)
     if (MODE != 2) {
         // ---- pass 1: the value of every tile ----
         {
-            const int t_lo = tile_lo + (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
-            int t_hi = t_lo + a.tiles_per_warp;
-            if (t_hi > tile_hi) t_hi = tile_hi;
+            const int t_lo = p_lo, t_hi = p_hi;
             if (t_lo < t_hi) {
                 // whole tiles pipelined; the row's ragged last tile (if it is this warp's) on its own
-                const int whole = a.v_p / OD_SAMPLE_TILE;
-                const int hi_w = t_hi < whole ? t_hi : whole;
+                const int hi_w = p_hi_w;
                 if (q.residual) {
-                    if (t_lo < hi_w) warp_tiles_dense_piped<DTYPE>(q, a, t_lo, hi_w, lane, tile_val);
+                    if (t_lo < hi_w) warp_tiles_dense_piped<DTYPE>(q, a, t_lo, hi_w, lane, tile_val, ni);
                     if (hi_w < t_hi) warp_tiles_dense<DTYPE, 2>(q, a, true, hi_w > t_lo ? hi_w : t_lo, t_hi, lane, tile_val);
                 } else {
                     warp_tiles_dense<DTYPE, 2>(q, a, false, t_lo, t_hi, lane, tile_val);
