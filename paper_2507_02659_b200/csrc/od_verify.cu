@@ -73,6 +73,8 @@ struct VerifyArgs {
     int32_t span_a;                     // units of space A per block
     int32_t a_early;                    // 1: space A is streamed before griddepcontrol.wait (the caller allows
                                         // it and a block's span of space A has at most A_PARK segments)
+    uint32_t w_mul, w_sh;               // n / W and n / n_chunks for n < 2^31 by multiplication (fast_div)
+    uint32_t c_mul, c_sh;
     const int32_t *tgt_ids;
     const float *q_prime;
     const int32_t *span_len;
@@ -266,6 +268,36 @@ __device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r,
     if (lane == 0) dst[warp] = make_float4(c, s, mx, 0.f);
 }
 
+// n / d for n < 2^31 and a divisor known at launch: with l = ceil(log2 d) and
+// mul = ceil(2^(31+l) / d) < 2^32, floor(n / d) = (n * mul) >> (31 + l) exactly, because
+// mul * d exceeds 2^(31+l) by less than d <= 2^l. mul == 0 stands for d == 1.
+__device__ __forceinline__ uint32_t div_by(uint32_t n, uint32_t mul, uint32_t sh)
+{
+    return mul ? __umulhi(n, mul) >> sh : n;
+}
+
+// Row rho of space B (rows 1..m_b of every sequence, in sequence order): its sequence b,
+// its row r and m_b. Lane l holds the sequences [i0, i1) and `excl`, the number of rows
+// of space B before them; exactly one lane finds rho among its own (rho < rows of space
+// B), and a shuffle tells the others. No shared memory and no barrier: a warp needs
+// nothing from the rest of its block.
+__device__ __forceinline__ void find_row(const VerifyArgs &a, uint32_t rho, int i0, int i1, uint32_t excl,
+                                         int &b, int &r, int &mb)
+{
+    uint32_t run = excl;
+    int hit = -1;
+#pragma unroll 4
+    for (int i = i0; i < i1; ++i) {
+        const uint32_t mi = (uint32_t)clamp_m(a.m[i], a.K_max);
+        if (rho - run < mi) hit = i | (int)(1u + rho - run) << 12 | (int)mi << 20;   // run <= rho < run + mi
+        run += mi;
+    }
+    const unsigned found = __ballot_sync(0xFFFFFFFFu, hit >= 0);
+    hit = __shfl_sync(0xFFFFFFFFu, hit, __ffs(found) - 1);
+    b = hit & 0xFFF; r = hit >> 12 & 0xFF; mb = hit >> 20;
+}
+static_assert(OD_VERIFY_MAX_B <= 4096 && OD_MAX_K < 255, "find_row packs (b, r, m_b) into one word");
+
 // first of the WARPS partial slots of segment `seg` of row (b, r)
 __device__ __forceinline__ float4 *partial_slot(const VerifyArgs &a, int b, int r, int seg)
 {
@@ -279,13 +311,14 @@ template <int DTYPE>
 __global__ void __maxnreg__(OD_VERIFY_MAXNREG)
 od_verify_stream_kernel(const VerifyArgs a)
 {
-    __shared__ int32_t s_cum[OD_VERIFY_MAX_B + 1];          // exclusive prefix of the clamped m_b
-    __shared__ int32_t s_wsum[WARPS];
     __shared__ float4 s_park[A_PARK][WARPS];
 
-    // Flat unit indices fit 32 bits (the launcher checks): the walk below is
-    // executed by every thread, so it uses 32-bit arithmetic and as few
-    // divisions as it can (one warp has only a few hundred useful instructions).
+    // Flat unit indices stay below 2^31 (the launcher checks). What a block does between
+    // griddepcontrol.wait and its first load of space B is the one stretch of this kernel
+    // in which the memory system has nothing to do, and with 32 warps per multiprocessor
+    // that run the same code every instruction there costs eight issue cycles: the
+    // walk below uses 32-bit arithmetic, multiplications in place of the divisions by W and
+    // by the grid size, registers and shuffles in place of shared memory and barriers.
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t g = blockIdx.x;
     const uint32_t W = (uint32_t)a.W;
@@ -301,7 +334,7 @@ od_verify_stream_kernel(const VerifyArgs a)
     if (a_lo > a_tot) a_lo = a_tot;
     uint32_t a_hi = a_lo + (uint32_t)a.span_a;
     if (a_hi > a_tot) a_hi = a_tot;
-    const uint32_t a_b0 = a_lo / W, a_v0 = a_lo - a_b0 * W;   // first sequence and unit of the span
+    const uint32_t a_b0 = div_by(a_lo, a.w_mul, a.w_sh), a_v0 = a_lo - a_b0 * W;   // first sequence and unit of the span
     const uint32_t a_seg0 = g - (a_lo - a_v0) / (uint32_t)a.span_a;   // a row that starts here has segment 0 here
     const bool early = a.a_early != 0;                      // the span has at most A_PARK segments
     if (early && a_lo < a_hi) {
@@ -314,87 +347,72 @@ od_verify_stream_kernel(const VerifyArgs a)
             f += n; ++b; v0 = 0;
         }
     }
+    // lane l of every warp will hold the sequences [i0, i1)
+    const int per = (a.B + 31) >> 5;
+    const int i0 = lane * per < a.B ? lane * per : a.B;
+    const int i1 = i0 + per < a.B ? i0 + per : a.B;
+    const uint32_t chunk = (uint32_t)a.n_chunks - 1 - g;    // spans of space B are handed out from the other end of the grid
 
     // everything below may read what the translation kernel wrote, and may write scratch
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
 
-    // ---- prefix sums of m (clamped) for space B
-    {
-        const int per = (a.B + THREADS - 1) / THREADS;
-        const int i0 = threadIdx.x * per;
-        int loc = 0;
-        for (int i = i0; i < i0 + per && i < a.B; ++i) loc += clamp_m(a.m[i], a.K_max);
-        int inc = loc;
+    // ---- rows of space B before each lane's sequences, and in all
+    uint32_t loc = 0;
+#pragma unroll 4
+    for (int i = i0; i < i1; ++i) loc += (uint32_t)clamp_m(a.m[i], a.K_max);
+    uint32_t inc = loc;
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int t = __shfl_up_sync(0xFFFFFFFFu, inc, off);
-            if (lane >= off) inc += t;
-        }
-        if (lane == 31) s_wsum[warp] = inc;
-        __syncthreads();
-        int base = 0;
-        for (int w = 0; w < warp; ++w) base += s_wsum[w];
-        int run = base + inc - loc;
-        for (int i = i0; i < i0 + per && i < a.B; ++i) {
-            s_cum[i] = run;
-            run += clamp_m(a.m[i], a.K_max);
-        }
-        if (threadIdx.x == THREADS - 1) s_cum[a.B] = base + inc;
-        __syncthreads();
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+        if (lane >= off) inc += t;
     }
+    const uint32_t rows_b = __shfl_sync(0xFFFFFFFFu, inc, 31);
+    const uint32_t excl = inc - loc;
 
-    if (a_lo < a_hi) {
-        if (early) {
-            // hand the parked partials over (the barriers above made them visible)
-            uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
-            int k = 0;
-            while (f < a_hi) {
-                uint32_t n = a_hi - f;
-                if (n > W - v0) n = W - v0;
-                if (warp == (k & (WARPS - 1)) && lane < WARPS)
-                    partial_slot(a, (int)b, 0, (int)seg)[lane] = s_park[k][lane];
-                ++k; f += n; ++b; v0 = 0; seg = 0;
-            }
-        } else {
-            uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
-            while (f < a_hi) {
-                uint32_t n = a_hi - f;
-                if (n > W - v0) n = W - v0;
-                block_segment<DTYPE>(a, (int)b, 0, (int)v0, (int)(v0 + n), partial_slot(a, (int)b, 0, (int)seg));
-                f += n; ++b; v0 = 0; seg = 0;
-            }
+    if (!early && a_lo < a_hi) {
+        uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
+        while (f < a_hi) {
+            uint32_t n = a_hi - f;
+            if (n > W - v0) n = W - v0;
+            block_segment<DTYPE>(a, (int)b, 0, (int)v0, (int)(v0 + n), partial_slot(a, (int)b, 0, (int)seg));
+            f += n; ++b; v0 = 0; seg = 0;
         }
     }
 
-    // ---- space B (rows 1..m_b), spans handed out from the other end of the grid
-    {
-        const uint32_t rows_b = (uint32_t)s_cum[a.B];
-        const uint32_t b_tot = rows_b * W;
-        if (b_tot == 0) return;
-        uint32_t span = (b_tot + (uint32_t)a.n_chunks - 1) / (uint32_t)a.n_chunks;
-        if (span < (uint32_t)a.span_min) span = (uint32_t)a.span_min;
-        const uint32_t chunk = (uint32_t)a.n_chunks - 1 - g;
-        uint32_t f = chunk * span;
-        if (f >= b_tot) return;
+    // ---- space B (rows 1..m_b)
+    const uint32_t b_tot = rows_b * W;
+    uint32_t span = div_by(b_tot + (uint32_t)a.n_chunks - 1, a.c_mul, a.c_sh);
+    if (span < (uint32_t)a.span_min) span = (uint32_t)a.span_min;
+    uint32_t f = chunk * span;
+    if (f < b_tot) {
         uint32_t f_hi = f + span;
         if (f_hi > b_tot) f_hi = b_tot;
-        uint32_t rho = f / W, v0 = f - rho * W;
+        uint32_t rho = div_by(f, a.w_mul, a.w_sh), v0 = f - rho * W;
         uint32_t seg = chunk - (f - v0) / span;
-        // sequence holding flat row rho: the last b with cum[b] <= rho (skips m_b = 0)
-        int lo = 0, hi = a.B;                                // invariant: cum[lo] <= rho < cum[hi]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if ((uint32_t)s_cum[mid] <= rho) lo = mid; else hi = mid;
-        }
-        int b = lo;
-        while (f < f_hi) {
-            while ((uint32_t)s_cum[b + 1] <= rho) ++b;
+        int b, r, mb;
+        find_row(a, rho, i0, i1, excl, b, r, mb);
+        for (;;) {
             uint32_t n = f_hi - f;
             if (n > W - v0) n = W - v0;
-            const int r = 1 + (int)(rho - (uint32_t)s_cum[b]);
             block_segment<DTYPE>(a, b, r, (int)v0, (int)(v0 + n), partial_slot(a, b, r, (int)seg));
-            f += n; ++rho; v0 = 0; seg = 0;
+            f += n;
+            if (f >= f_hi) break;
+            ++rho; v0 = 0; seg = 0;
+            if (r < mb) ++r; else find_row(a, rho, i0, i1, excl, b, r, mb);
+        }
+    }
+
+    // ---- the parked partials of space A: every warp hands over its own (its lane 0
+    // wrote them), at the end, where nothing waits for it
+    if (early && a_lo < a_hi && lane == 0) {
+        uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
+        int k = 0;
+        while (f < a_hi) {
+            uint32_t n = a_hi - f;
+            if (n > W - v0) n = W - v0;
+            partial_slot(a, (int)b, 0, (int)seg)[warp] = s_park[k][warp];
+            ++k; f += n; ++b; v0 = 0; seg = 0;
         }
     }
 }
@@ -593,6 +611,17 @@ cudaError_t launch(Kern kern, unsigned grid, unsigned block, cudaStream_t s, boo
 
 }  // namespace
 
+// multiplier and shift of div_by for the divisor d >= 1
+static void fast_div(uint32_t d, uint32_t &mul, uint32_t &sh)
+{
+    if (d <= 1) { mul = 0; sh = 0; return; }
+    uint32_t l = 0;
+    while (((uint64_t)1 << l) < d) ++l;                     // l = ceil(log2 d) >= 1
+    const unsigned __int128 num = (unsigned __int128)1 << (31 + l);
+    mul = (uint32_t)((num + d - 1) / d);
+    sh = l - 1;
+}
+
 // Launch plan of the stream kernel for `nb` sequences whose rows hold `v_len` elements.
 static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_len, int32_t dtype, bool early,
                         VerifyArgs &a)
@@ -615,6 +644,8 @@ static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_le
     if (span_a < span_min) span_a = span_min;
     a.span_a = (int32_t)span_a;
     a.a_early = early && span_a / W + 2 <= A_PARK;
+    fast_div((uint32_t)W, a.w_mul, a.w_sh);
+    fast_div((uint32_t)grid, a.c_mul, a.c_sh);
 }
 
 // batches beyond the shared-memory prefix table go in slices; a slice's flat
