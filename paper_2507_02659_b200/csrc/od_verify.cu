@@ -282,15 +282,22 @@ __device__ __forceinline__ uint32_t div_by(uint32_t n, uint32_t mul, uint32_t sh
 // B), and a shuffle tells the others. No shared memory and no barrier: a warp needs
 // nothing from the rest of its block.
 __device__ __forceinline__ void find_row(const VerifyArgs &a, uint32_t rho, int i0, int i1, uint32_t excl,
-                                         int &b, int &r, int &mb)
+                                         uint32_t m0, uint32_t m1, int &b, int &r, int &mb)
 {
     uint32_t run = excl;
     int hit = -1;
+    if (i1 - i0 <= 2) {
+        // the lane's (clamped) m are in registers: m0, m1 (0 where the lane has no sequence)
+        if (rho - run < m0) hit = i0 | (int)(1u + rho - run) << 12 | (int)m0 << 20;
+        run += m0;
+        if (rho - run < m1) hit = (i0 + 1) | (int)(1u + rho - run) << 12 | (int)m1 << 20;
+    } else {
 #pragma unroll 4
-    for (int i = i0; i < i1; ++i) {
-        const uint32_t mi = (uint32_t)clamp_m(a.m[i], a.K_max);
-        if (rho - run < mi) hit = i | (int)(1u + rho - run) << 12 | (int)mi << 20;   // run <= rho < run + mi
-        run += mi;
+        for (int i = i0; i < i1; ++i) {
+            const uint32_t mi = (uint32_t)clamp_m(a.m[i], a.K_max);
+            if (rho - run < mi) hit = i | (int)(1u + rho - run) << 12 | (int)mi << 20;   // run <= rho < run + mi
+            run += mi;
+        }
     }
     const unsigned found = __ballot_sync(0xFFFFFFFFu, hit >= 0);
     hit = __shfl_sync(0xFFFFFFFFu, hit, __ffs(found) - 1);
@@ -358,9 +365,15 @@ od_verify_stream_kernel(const VerifyArgs a)
     asm volatile("griddepcontrol.launch_dependents;");
 
     // ---- rows of space B before each lane's sequences, and in all
-    uint32_t loc = 0;
+    uint32_t loc = 0, m0 = 0, m1 = 0;
+    if (i1 - i0 <= 2) {
+        if (i0 < i1) m0 = (uint32_t)clamp_m(a.m[i0], a.K_max);
+        if (i0 + 1 < i1) m1 = (uint32_t)clamp_m(a.m[i0 + 1], a.K_max);
+        loc = m0 + m1;
+    } else {
 #pragma unroll 4
-    for (int i = i0; i < i1; ++i) loc += (uint32_t)clamp_m(a.m[i], a.K_max);
+        for (int i = i0; i < i1; ++i) loc += (uint32_t)clamp_m(a.m[i], a.K_max);
+    }
     uint32_t inc = loc;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -391,7 +404,7 @@ od_verify_stream_kernel(const VerifyArgs a)
         uint32_t rho = div_by(f, a.w_mul, a.w_sh), v0 = f - rho * W;
         uint32_t seg = chunk - (f - v0) / span;
         int b, r, mb;
-        find_row(a, rho, i0, i1, excl, b, r, mb);
+        find_row(a, rho, i0, i1, excl, m0, m1, b, r, mb);
         for (;;) {
             uint32_t n = f_hi - f;
             if (n > W - v0) n = W - v0;
@@ -399,7 +412,7 @@ od_verify_stream_kernel(const VerifyArgs a)
             f += n;
             if (f >= f_hi) break;
             ++rho; v0 = 0; seg = 0;
-            if (r < mb) ++r; else find_row(a, rho, i0, i1, excl, b, r, mb);
+            if (r < mb) ++r; else find_row(a, rho, i0, i1, excl, m0, m1, b, r, mb);
         }
     }
 
