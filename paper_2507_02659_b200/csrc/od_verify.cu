@@ -189,6 +189,24 @@ __device__ __forceinline__ void absorb_one(Lane<DTYPE> &L, float x, float scale)
     L.s += od_ex2(fmaf(x, scale, -L.c));
 }
 
+// the first n (1..U, the same for the whole warp) loads of a group
+__device__ __forceinline__ void load_group(uint4 (&x)[U], const uint4 *p, int n)
+{
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+        if (u < n) x[u] = ld_stream(p + u * WARPS * 32);
+}
+
+template <int DTYPE>
+__device__ __forceinline__ void absorb_group(Lane<DTYPE> &L, const uint4 (&x)[U], int n, float scale)
+{
+    static_assert(U == 4, "one case per group size");
+    if (n == 4) absorb<DTYPE, 4>(L, x, scale);
+    else if (n == 3) absorb<DTYPE, 3>(L, x, scale);
+    else if (n == 2) absorb<DTYPE, 2>(L, x, scale);
+    else absorb<DTYPE, 1>(L, x, scale);
+}
+
 // Units [v0, v1) of row (b, r) by the whole block; warp w stores its partial to dst[w]
 // (global or shared memory).
 template <int DTYPE>
@@ -202,53 +220,36 @@ __device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r,
     Lane<DTYPE> L;
     L.reset();
     // A warp owns whole units (512 bytes, 16 per lane): units v0 + warp, + WARPS, ...
-    // Groups of U units; what is left (1..U-1 units) takes a group of its own
-    // size, so no lane ever computes on padding. Only the row's last unit can be
-    // ragged (lanes past the end of the row, or a final piece under 16 bytes).
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int full_vecs = a.v_p / VEC;                     // whole 16-byte vectors in the row
     const int full_units = full_vecs >> 5;                 // units whose 32 lanes are all inside
     const int v1f = v1 < full_units ? v1 : full_units;
-    int v = v0 + warp;
+    const int v = v0 + warp;
     const uint4 *p = (const uint4 *)row + (size_t)v * 32 + lane;
     // Software pipeline over groups of U units: the loads of the next group are
     // issued before the current group is folded in, so a warp always has loads in
     // flight while it keeps the exp pipe busy (warps of a block move in lockstep,
-    // they cannot hide one another's latency).
-    if (v + (U - 1) * WARPS < v1f) {
+    // they cannot hide one another's latency). The last group holds what is left
+    // (1..U units) and is requested like any other, one group ahead; no lane ever
+    // computes on padding. Only the row's last unit can be ragged (lanes past the
+    // end of the row, or a final piece under 16 bytes).
+    int cnt = v < v1f ? (v1f - v + WARPS - 1) / WARPS : 0;   // this warp's whole units
+    if (cnt > 0) {
         uint4 xa[U], xb[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) xa[u] = ld_stream(p + u * WARPS * 32);
-        v += U * WARPS; p += U * WARPS * 32;
+        int na = cnt < U ? cnt : U, nb = 0;
+        load_group(xa, p, na);
+        cnt -= na; p += U * WARPS * 32;
         for (;;) {
-            if (!(v + (U - 1) * WARPS < v1f)) { absorb<DTYPE, U>(L, xa, scale); break; }
-#pragma unroll
-            for (int u = 0; u < U; ++u) xb[u] = ld_stream(p + u * WARPS * 32);
-            v += U * WARPS; p += U * WARPS * 32;
+            if (cnt == 0) { absorb_group<DTYPE>(L, xa, na, scale); break; }
+            nb = cnt < U ? cnt : U;
+            load_group(xb, p, nb);
+            cnt -= nb; p += U * WARPS * 32;
             absorb<DTYPE, U>(L, xa, scale);
-            if (!(v + (U - 1) * WARPS < v1f)) { absorb<DTYPE, U>(L, xb, scale); break; }
-#pragma unroll
-            for (int u = 0; u < U; ++u) xa[u] = ld_stream(p + u * WARPS * 32);
-            v += U * WARPS; p += U * WARPS * 32;
+            if (cnt == 0) { absorb_group<DTYPE>(L, xb, nb, scale); break; }
+            na = cnt < U ? cnt : U;
+            load_group(xa, p, na);
+            cnt -= na; p += U * WARPS * 32;
             absorb<DTYPE, U>(L, xb, scale);
-        }
-    }
-    if (v < v1f) {
-        const int left = (v1f - v + WARPS - 1) / WARPS;    // 1..U-1, the same for the whole warp
-        if (left == 3) {
-            uint4 x[3];
-#pragma unroll
-            for (int u = 0; u < 3; ++u) x[u] = ld_stream(p + u * WARPS * 32);
-            absorb<DTYPE, 3>(L, x, scale);
-        } else if (left == 2) {
-            uint4 x[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) x[u] = ld_stream(p + u * WARPS * 32);
-            absorb<DTYPE, 2>(L, x, scale);
-        } else {
-            uint4 x[1];
-            x[0] = ld_stream(p);
-            absorb<DTYPE, 1>(L, x, scale);
         }
     }
     if (v1 > full_units && warp == ((full_units - v0) & (WARPS - 1))) {
