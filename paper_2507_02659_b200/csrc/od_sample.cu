@@ -376,21 +376,35 @@ od_sample_kernel(const SampleArgs a)
     // (a.early = 0: the launch before this one was not od_verify; everything waits.)
     asm volatile("griddepcontrol.launch_dependents;");
     if (!a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Two memory round trips, not a chain of four: everything that is addressed by (b, lane)
+    // alone is requested at once, whether or not it will be used (lane < K keeps the
+    // addresses inside the arrays); what is addressed by those values comes second.
     int mb = a.m[b];
-    mb = mb < 0 ? 0 : (mb > K ? K : mb);
     const bool stop = a.tail_kind[b] == OD_TAIL_UNMAPPED_STOP;
     const float T = a.temperature[b];
+    int32_t l_s0 = 0, l_len = 1, l_tgt = -1, l_did = -1;
+    float l_qp = 0.f;
+    if (lane < K) {
+        const size_t o = (size_t)b * K + lane;
+        l_s0 = a.span_start[o];
+        l_len = a.span_len[o];
+        l_tgt = a.tgt_ids[o];
+        l_qp = a.q_prime[o];
+        l_did = a.draft_ids[o];
+    }
+    mb = mb < 0 ? 0 : (mb > K ? K : mb);
     int32_t e_s0 = 0, e_len = 1, e_tgt = -1, e_d1 = -1, e_pm = -1;
     float e_qp = 0.f, e_qd1 = 0.f;
-    if (lane < K && lane <= mb) {
-        const size_t o = (size_t)b * K + lane;
-        int s0 = a.span_start[o];
-        e_s0 = s0 < 0 ? 0 : (s0 >= K ? K - 1 : s0);
-        e_len = lane < mb ? a.span_len[o] : 1;
-        if (e_len >= 2) {
-            e_tgt = a.tgt_ids[o];
-            e_qp = a.q_prime[o];
-            const int32_t d1 = a.draft_ids[(size_t)b * K + e_s0];
+    {
+        const bool live = lane < K && lane <= mb;
+        if (live) {
+            e_s0 = l_s0 < 0 ? 0 : (l_s0 >= K ? K - 1 : l_s0);
+            e_len = lane < mb ? l_len : 1;
+        }
+        const int32_t d1 = __shfl_sync(0xFFFFFFFFu, l_did, e_s0);   // the span's first draft token
+        if (live && e_len >= 2) {
+            e_tgt = l_tgt;
+            e_qp = l_qp;
             if (d1 >= 0 && d1 < a.v_q) {
                 e_d1 = d1;
                 e_pm = __ldg(a.vocab_map + d1);
@@ -419,15 +433,14 @@ od_sample_kernel(const SampleArgs a)
         if (lane == 0) { s_red[0][warp] = before; s_red[1][warp] = total; }
         if (threadIdx.x == 0) s_vbits = 0;
         if (lane < mb) {
-            const size_t o = (size_t)b * K + lane;
-            const int32_t t = a.tgt_ids[o];
+            const int32_t t = l_tgt;
             d_tok = t >= 0 && t < a.v_p;
             const char *row_k = (const char *)a.logits +
                                 ((size_t)b * a.seq_stride + (size_t)lane * a.row_stride) * (DTYPE == OD_BF16 ? 2 : 4);
             if (d_tok) d_xt = od_load_logit<DTYPE>(row_k, t);
-            d_q = a.q_prime[o];
+            d_q = l_qp;
             d_u = od_uniform(a.seed[b], a.step, (uint32_t)lane, 0u);
-            d_span = a.span_len[o];
+            d_span = l_len;
         }
         __syncthreads();
         before = 0; total = 0;
