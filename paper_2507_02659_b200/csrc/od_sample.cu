@@ -356,7 +356,6 @@ od_sample_kernel(const SampleArgs a)
 {
     __shared__ float s_M[FUSED ? OD_MAX_K + 1 : 1], s_S[FUSED ? OD_MAX_K + 1 : 1];
     __shared__ int s_red[2][WARPS];
-    __shared__ int s_n;
     __shared__ unsigned int s_vbits;
     extern __shared__ __align__(16) unsigned char s_dyn[];   // ntiles x 8 bytes
     double *s_val = (double *)s_dyn;                         // pass 2: tile values
@@ -461,6 +460,7 @@ od_sample_kernel(const SampleArgs a)
     // n_accepted and the row statistics come from the verification kernels
     if (a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
 
+    int fused_n = 0;
     if (FUSED) {
         // ---- step 2's decisions (what od_verify_decide_kernel does, same arithmetic, same order)
         const bool bad_T = !(T > 0.f);
@@ -477,28 +477,34 @@ od_sample_kernel(const SampleArgs a)
             }
         }
         __syncthreads();
-        if (warp == 0) {
+        // every warp takes the decisions for itself (lane k = position k holds the inputs in
+        // every warp): no second barrier; warp 0 of the sequence's first block stores them
+        int n = 0;
+        {
             bool acc = false, bnd = false;
+            Acceptance d = {};
             if (lane < mb) {
-                const Acceptance d = accept_position(s_M[lane], s_S[lane], dscale, d_tok, d_xt, d_q, d_u);
+                d = accept_position(s_M[lane], s_S[lane], dscale, d_tok, d_xt, d_q, d_u);
                 acc = d.accept; bnd = d.boundary;
-                if (blockIdx.x == 0) { a.w_p_sel[(size_t)b * K + lane] = d.p; a.w_ratio[(size_t)b * K + lane] = d.ratio; }
             }
-            const unsigned int accmask = __ballot_sync(0xFFFFFFFFu, acc), bndmask = __ballot_sync(0xFFFFFFFFu, bnd);
-            int n = 0;
+            const unsigned int accmask = __ballot_sync(0xFFFFFFFFu, acc);
             while (n < mb && (accmask >> n & 1u)) ++n;
-            int nd = lane < n ? d_span : 0;
+            if (bad_T) n = 0;
+            if (blockIdx.x == 0 && warp == 0) {
+                if (lane < mb) { a.w_p_sel[(size_t)b * K + lane] = d.p; a.w_ratio[(size_t)b * K + lane] = d.ratio; }
+                const unsigned int bndmask = __ballot_sync(0xFFFFFFFFu, bnd);
+                int nd = lane < n ? d_span : 0;
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) nd += __shfl_xor_sync(0xFFFFFFFFu, nd, off);
-            if (lane == 0) {
-                uint32_t f = bndmask & OD_VF_BOUNDARY_MASK;
-                if (s_vbits & 1u) f |= OD_VF_NONFINITE;
-                if (bad_T) { f |= OD_VF_BAD_TEMPERATURE; n = 0; nd = 0; }
-                s_n = n;
-                if (blockIdx.x == 0) { a.w_n_accepted[b] = n; a.w_n_draft[b] = nd; a.w_vflags[b] = f; }
+                for (int off = 16; off > 0; off >>= 1) nd += __shfl_xor_sync(0xFFFFFFFFu, nd, off);
+                if (lane == 0) {
+                    uint32_t f = bndmask & OD_VF_BOUNDARY_MASK;
+                    if (s_vbits & 1u) f |= OD_VF_NONFINITE;
+                    if (bad_T) f |= OD_VF_BAD_TEMPERATURE;
+                    a.w_n_accepted[b] = n; a.w_n_draft[b] = nd; a.w_vflags[b] = f;
+                }
             }
         }
-        __syncthreads();
+        fused_n = n;
     }
 
     if (!(T > 0.f)) {                              // every block of the sequence leaves here
@@ -516,7 +522,7 @@ od_sample_kernel(const SampleArgs a)
         rm = FUSED ? s_M[lane] : a.row_max[b * (K + 1) + lane];
         rs = FUSED ? s_S[lane] : a.row_sum[b * (K + 1) + lane];
     }
-    int j = FUSED ? s_n : a.n_accepted[b];
+    int j = FUSED ? fused_n : a.n_accepted[b];
     j = j < 0 ? 0 : (j > mb ? mb : j);
     const size_t esz = DTYPE == OD_BF16 ? 2 : 4;
     // a shard's row pointer is moved back by the shard's first column, and only ids of
