@@ -41,13 +41,18 @@
  *     wait in two cases only: inside od_step / od_step_host, where the
  *     translation kernel is the launch in front of the streaming kernel and has
  *     itself waited for everything earlier in the stream before letting it
- *     start; and in od_verify when the caller has set option "early_inputs" = 1,
- *     which is the caller's promise that the step's inputs were complete before
- *     the launch that precedes the call was enqueued (a producer two launches
- *     back, or data resident since an earlier synchronisation). A producer that
- *     is the launch directly in front of od_verify (the target model's output
- *     layer, say) is always safe with the default "early_inputs" = 0.
- *     "pdl" = 0 gives plain stream order.
+ *     start (logits and temperatures, by the streaming kernel); and when the
+ *     caller has set option "early_inputs" = 1, which is the caller's promise
+ *     that the inputs of a call were complete before the launch that precedes
+ *     the call was enqueued (a producer two launches back, or data resident
+ *     since an earlier synchronisation): then od_verify and
+ *     od_verify_shard_stats read logits and temperatures early, and
+ *     od_map_proposals and od_step read the proposal (draft ids, lengths,
+ *     q_sel) early; the n-gram table is never read early. A producer that is
+ *     the launch directly in front of a call (the target model's output layer,
+ *     the drafter's sampling kernel) is always safe with the default
+ *     "early_inputs" = 0. od_step_host copies its inputs itself and reads
+ *     nothing of the caller's early. "pdl" = 0 gives plain stream order.
  *   - Positions: arrays indexed [B, K_max] hold K_max entries per sequence,
  *     of which the first K_b (inputs) or m_b (outputs) are meaningful.
  *   - Random numbers: Philox4x32-10 (Salmon et al., SC'11) with key = the
@@ -211,8 +216,9 @@ int32_t od_cache_dump(od_ctx *ctx, int64_t max_out, int32_t *runs, int32_t *len,
 /* Options. Names: "pdl" (1 = launch the step kernels with programmatic stream
  * serialization so that a kernel's prologue overlaps its predecessor's tail, the
  * default; 0 = plain stream order), "early_inputs" (1 = od_verify and
- * od_verify_shard_stats may read logits and temperatures before they wait for the
- * launch in front of them, see the conventions above; default 0),
+ * od_verify_shard_stats may read logits and temperatures, od_map_proposals and
+ * od_step the proposal, before they wait for the launch in front of them, see the
+ * conventions above; default 0),
  * "verify_grid" (thread blocks of od_verify's streaming kernel, 0 = one per
  * multiprocessor, the default), "sample_tiles_per_warp" (256-id tiles one warp of
  * od_sample_residual sums, 0 = automatic). Unknown name: INVALID_ARG. */

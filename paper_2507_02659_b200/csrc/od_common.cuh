@@ -55,7 +55,8 @@ struct od_ctx {
 
     // options
     int64_t opt_verify_grid;        // blocks of the stream kernel (0 = one per multiprocessor)
-    int64_t opt_early_inputs;       // od_verify may read logits and temperatures before griddepcontrol.wait
+    int64_t opt_early_inputs;       // the caller promises complete inputs: od_verify reads logits and temperatures, the
+                                    // translation kernel the proposal, before griddepcontrol.wait
     int64_t opt_sample_tiles_per_warp;
     int64_t opt_pdl;                // launch with programmatic stream serialization
 
@@ -86,7 +87,7 @@ struct od_ctx {
 cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids,
                           const int32_t *draft_len, const float *q_sel, int32_t *tgt_ids,
                           float *q_prime, int32_t *span_start, int32_t *span_len, int32_t *m,
-                          uint8_t *tail_kind, uint32_t *counters, cudaStream_t s);
+                          uint8_t *tail_kind, uint32_t *counters, bool early, cudaStream_t s);
 
 cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
                              int32_t dtype, int64_t row_stride, int64_t seq_stride,

@@ -46,7 +46,7 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
               float *__restrict__ q_prime, int32_t *__restrict__ span_start,
               int32_t *__restrict__ span_len, int32_t *__restrict__ m_out,
               uint8_t *__restrict__ tail_kind, uint32_t *__restrict__ counters,
-              uint32_t *__restrict__ stamp, uint32_t *__restrict__ freq, uint32_t clock)
+              uint32_t *__restrict__ stamp, uint32_t *__restrict__ freq, uint32_t clock, int32_t early)
 {
     __shared__ int32_t s_ids[OD_MAX_K];
     __shared__ int32_t s_hit[OD_MAX_K][OD_NGRAM_MAX + 1];   // [offset][length] -> target or -1
@@ -54,18 +54,34 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
     __shared__ int32_t s_direct[OD_MAX_K];                  // direct map of the id at each offset, or -1
     __shared__ float s_q[OD_MAX_K];                         // q(d) of each offset
 
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // The proposal itself (ids, length, probabilities) is the caller's input. Where the
+    // caller has promised that it was complete before the launch in front of this one was
+    // enqueued (early), it is requested before the wait; the table and everything this
+    // kernel writes always wait.
+    int K = 0;
+    int32_t my_id = -1;
+    float my_q = 0.f;
+    if (early && b < B) {
+        K = draft_len[b];
+        if (threadIdx.x < K_max) my_id = draft_ids[(size_t)b * K_max + threadIdx.x];
+        if (lane == 0 && warp < K_max) my_q = q_sel[(size_t)b * K_max + warp];
+    }
+
     // under programmatic dependent launch: wait for everything earlier in the
     // stream first, only then let the verification kernel start its prefetch
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
 
-    const int b = blockIdx.x;
     if (b >= B) return;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int K = draft_len[b];
+    if (!early) {
+        K = draft_len[b];
+        if (threadIdx.x < K_max) my_id = draft_ids[(size_t)b * K_max + threadIdx.x];
+        if (lane == 0 && warp < K_max) my_q = q_sel[(size_t)b * K_max + warp];
+    }
     K = K < 0 ? 0 : (K > K_max ? K_max : K);
-
-    if (threadIdx.x < K_max) s_ids[threadIdx.x] = draft_ids[(size_t)b * K_max + threadIdx.x];
+    if (threadIdx.x < K_max) s_ids[threadIdx.x] = my_id;
     __syncthreads();
 
     const int s = warp;
@@ -74,7 +90,7 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
         if (lane == 0) {
             const int32_t id = s_ids[s];
             s_direct[s] = (id >= 0 && id < v_q) ? __ldg(vocab_map + id) : -1;
-            s_q[s] = q_sel[(size_t)b * K_max + s];
+            s_q[s] = my_q;
         }
         int32_t hit[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
         int32_t slot[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
@@ -170,7 +186,7 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
 cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids,
                           const int32_t *draft_len, const float *q_sel, int32_t *tgt_ids,
                           float *q_prime, int32_t *span_start, int32_t *span_len, int32_t *m,
-                          uint8_t *tail_kind, uint32_t *counters, cudaStream_t s)
+                          uint8_t *tail_kind, uint32_t *counters, bool early, cudaStream_t s)
 {
     if (B == 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
@@ -187,5 +203,5 @@ cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *dr
                               (const int32_t *)c->d_vocab_map, (const uint64_t *)c->d_keys,
                               (const int32_t *)c->d_vals, c->cap, tgt_ids, q_prime, span_start,
                               span_len, m, tail_kind, counters, c->dyn ? c->d_stamp : (uint32_t *)nullptr,
-                              c->dyn ? c->d_freq : (uint32_t *)nullptr, c->clock);
+                              c->dyn ? c->d_freq : (uint32_t *)nullptr, c->clock, (int32_t)(early && c->opt_pdl));
 }

@@ -300,6 +300,19 @@ def test_od_step_equals_the_three_calls(cuda_device):
     assert torch.equal(vo.flags, vo2.flags)
     assert torch.equal(so.out_token, so2.out_token) and torch.equal(so.flags, so2.flags)
     assert torch.equal(so.resid_mass, so2.resid_mass)
+    # inputs that have been resident since a synchronisation: the caller may promise so
+    # ("early_inputs"), and then the translation kernel reads the proposal before it waits
+    # for the sampler of the step in front. Steps back to back, same bits.
+    ctx.set_option("early_inputs", 1)
+    torch.cuda.synchronize()
+    runs = [od.od_step(ctx, s.draft_ids, s.draft_len, s.q_sel, s.q_rows, lg, s.temperature, s.seed, s.step)
+            for _ in range(6)]
+    torch.cuda.synchronize()
+    for mp3, vo3, so3 in runs:
+        assert torch.equal(mp.m, mp3.m) and torch.equal(mp.tgt_ids[pos], mp3.tgt_ids[pos])
+        assert torch.equal(mp.q_prime[pos], mp3.q_prime[pos]) and torch.equal(mp.tail_kind, mp3.tail_kind)
+        assert torch.equal(vo.row_sum[rows], vo3.row_sum[rows]) and torch.equal(vo.n_accepted, vo3.n_accepted)
+        assert torch.equal(so.out_token, so3.out_token) and torch.equal(so.resid_mass, so3.resid_mass)
     ctx.close()
 
 
