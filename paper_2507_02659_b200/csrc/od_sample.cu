@@ -606,12 +606,27 @@ od_sample_kernel(const SampleArgs a)
     // ---- pass 2 (one block per sequence) ----
     bool residual = q.residual;
     uint32_t flags = residual ? 0u : OD_SF_BONUS;
-    const float u = MODE == 1 ? 0.f : od_uniform(a.seed[b], a.step, (uint32_t)j, 1u);
     const int per = (tile_hi - tile_lo + OD_SAMPLE_THREADS - 1) / OD_SAMPLE_THREADS;
     const int my_lo = tile_lo + threadIdx.x * per < tile_hi ? tile_lo + threadIdx.x * per : tile_hi;
     const int my_hi = my_lo + per < tile_hi ? my_lo + per : tile_hi;
-    // tile values (rounding can leave a tile without residual mass slightly negative)
-    for (int t = tile_lo + threadIdx.x; t < tile_hi; t += OD_SAMPLE_THREADS) s_val[t] = fmax(0.0, __ldcg(tile_val + t));
+    // tile values (rounding can leave a tile without residual mass slightly negative): four
+    // requests per thread at a time, and the draw's uniform worked out while they travel
+    float u = 0.f;
+    const uint64_t seed_b = MODE == 1 ? 0ull : a.seed[b];   // requested with the tile values, used behind them
+    for (int t0 = tile_lo + threadIdx.x, first = 1; first || t0 < tile_hi; t0 += 4 * OD_SAMPLE_THREADS, first = 0) {
+        double v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int t = t0 + i * OD_SAMPLE_THREADS;
+            v[i] = t < tile_hi ? __ldcg(tile_val + t) : 0.0;
+        }
+        if (MODE != 1 && first) u = od_uniform(seed_b, a.step, (uint32_t)j, 1u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int t = t0 + i * OD_SAMPLE_THREADS;
+            if (t < tile_hi) s_val[t] = fmax(0.0, v[i]);
+        }
+    }
     if (MODE != 2 && threadIdx.x == 0) a.ticket[b] = 0;
     __syncthreads();
 
