@@ -280,22 +280,23 @@ __device__ __forceinline__ uint32_t div_by(uint32_t n, uint32_t mul, uint32_t sh
 // Row rho of space B (rows 1..m_b of every sequence, in sequence order): its sequence b,
 // its row r and m_b. Lane l holds the sequences [i0, i1) and `excl`, the number of rows
 // of space B before them; exactly one lane finds rho among its own (rho < rows of space
-// B), and a shuffle tells the others. No shared memory and no barrier: a warp needs
-// nothing from the rest of its block.
-__device__ __forceinline__ void find_row(const VerifyArgs &a, uint32_t rho, int i0, int i1, uint32_t excl,
+// B), and a shuffle tells the others. With at most two sequences per lane their m are in
+// registers (m0, m1): no shared memory and no barrier, a warp needs nothing from the rest
+// of its block; larger batches read the block's copy s_m.
+__device__ __forceinline__ void find_row(const int32_t *s_m, uint32_t rho, int i0, int i1, uint32_t excl,
                                          uint32_t m0, uint32_t m1, int &b, int &r, int &mb)
 {
     uint32_t run = excl;
     int hit = -1;
-    if (i1 - i0 <= 2) {
+    if (s_m == nullptr) {
         // the lane's (clamped) m are in registers: m0, m1 (0 where the lane has no sequence)
         if (rho - run < m0) hit = i0 | (int)(1u + rho - run) << 12 | (int)m0 << 20;
         run += m0;
         if (rho - run < m1) hit = (i0 + 1) | (int)(1u + rho - run) << 12 | (int)m1 << 20;
     } else {
-#pragma unroll 4
+#pragma unroll 1
         for (int i = i0; i < i1; ++i) {
-            const uint32_t mi = (uint32_t)clamp_m(a.m[i], a.K_max);
+            const uint32_t mi = s_m[i];
             if (rho - run < mi) hit = i | (int)(1u + rho - run) << 12 | (int)mi << 20;   // run <= rho < run + mi
             run += mi;
         }
@@ -304,7 +305,23 @@ __device__ __forceinline__ void find_row(const VerifyArgs &a, uint32_t rho, int 
     hit = __shfl_sync(0xFFFFFFFFu, hit, __ffs(found) - 1);
     b = hit & 0xFFF; r = hit >> 12 & 0xFF; mb = hit >> 20;
 }
-static_assert(OD_VERIFY_MAX_B <= 4096 && OD_MAX_K < 255, "find_row packs (b, r, m_b) into one word");
+static_assert(OD_VERIFY_MAX_B <= 4096 && OD_MAX_K < 255 && OD_MAX_K <= 255, "find_row packs (b, r, m_b) into one word");
+
+// Block g's span of space A (row 0 of every sequence, W units each, span_a units per block):
+// flat units [lo, hi), the first one being unit v0 of sequence b0; a row that starts in the
+// span has its segment 0 here, the row the span starts inside has segment seg0 here.
+__device__ __forceinline__ void span_of_space_a(const VerifyArgs &a, uint32_t g, uint32_t &lo, uint32_t &hi,
+                                                uint32_t &b0, uint32_t &v0, uint32_t &seg0)
+{
+    const uint32_t W = (uint32_t)a.W, tot = (uint32_t)a.B * W;
+    lo = g * (uint32_t)a.span_a;
+    if (lo > tot) lo = tot;
+    hi = lo + (uint32_t)a.span_a;
+    if (hi > tot) hi = tot;
+    b0 = div_by(lo, a.w_mul, a.w_sh);
+    v0 = lo - b0 * W;
+    seg0 = g - (lo - v0) / (uint32_t)a.span_a;
+}
 
 // first of the WARPS partial slots of segment `seg` of row (b, r)
 __device__ __forceinline__ float4 *partial_slot(const VerifyArgs &a, int b, int r, int seg)
@@ -320,6 +337,7 @@ __global__ void __maxnreg__(OD_VERIFY_MAXNREG)
 od_verify_stream_kernel(const VerifyArgs a)
 {
     __shared__ float4 s_park[A_PARK][WARPS];
+    __shared__ int32_t s_m[OD_VERIFY_MAX_B];               // clamped m_b, batches of more than 64 sequences only
 
     // Flat unit indices stay below 2^31 (the launcher checks). What a block does between
     // griddepcontrol.wait and its first load of space B is the one stretch of this kernel
@@ -337,13 +355,8 @@ od_verify_stream_kernel(const VerifyArgs a)
     // while the launch in front is still at work. Its partials wait in shared memory: the
     // scratch in global memory may still be read by the previous launch's decide kernel
     // until griddepcontrol.wait returns.
-    const uint32_t a_tot = (uint32_t)a.B * W;
-    uint32_t a_lo = g * (uint32_t)a.span_a;
-    if (a_lo > a_tot) a_lo = a_tot;
-    uint32_t a_hi = a_lo + (uint32_t)a.span_a;
-    if (a_hi > a_tot) a_hi = a_tot;
-    const uint32_t a_b0 = div_by(a_lo, a.w_mul, a.w_sh), a_v0 = a_lo - a_b0 * W;   // first sequence and unit of the span
-    const uint32_t a_seg0 = g - (a_lo - a_v0) / (uint32_t)a.span_a;   // a row that starts here has segment 0 here
+    uint32_t a_lo, a_hi, a_b0, a_v0, a_seg0;
+    span_of_space_a(a, g, a_lo, a_hi, a_b0, a_v0, a_seg0);
     const bool early = a.a_early != 0;                      // the span has at most A_PARK segments
     if (early && a_lo < a_hi) {
         uint32_t f = a_lo, b = a_b0, v0 = a_v0;
@@ -367,13 +380,17 @@ od_verify_stream_kernel(const VerifyArgs a)
 
     // ---- rows of space B before each lane's sequences, and in all
     uint32_t loc = 0, m0 = 0, m1 = 0;
-    if (i1 - i0 <= 2) {
+    if (per <= 2) {
         if (i0 < i1) m0 = (uint32_t)clamp_m(a.m[i0], a.K_max);
         if (i0 + 1 < i1) m1 = (uint32_t)clamp_m(a.m[i0 + 1], a.K_max);
         loc = m0 + m1;
     } else {
-#pragma unroll 4
-        for (int i = i0; i < i1; ++i) loc += (uint32_t)clamp_m(a.m[i], a.K_max);
+        // more than 64 sequences: the block reads m once into shared memory (a load that is
+        // repeated goes to L2 again, and a warp looks its rows up once per sequence)
+        for (int i = threadIdx.x; i < a.B; i += THREADS) s_m[i] = clamp_m(a.m[i], a.K_max);
+        __syncthreads();
+#pragma unroll 1
+        for (int i = i0; i < i1; ++i) loc += (uint32_t)s_m[i];
     }
     uint32_t inc = loc;
 #pragma unroll
@@ -405,7 +422,7 @@ od_verify_stream_kernel(const VerifyArgs a)
         uint32_t rho = div_by(f, a.w_mul, a.w_sh), v0 = f - rho * W;
         uint32_t seg = chunk - (f - v0) / span;
         int b, r, mb;
-        find_row(a, rho, i0, i1, excl, m0, m1, b, r, mb);
+        find_row(per <= 2 ? nullptr : s_m, rho, i0, i1, excl, m0, m1, b, r, mb);
         for (;;) {
             uint32_t n = f_hi - f;
             if (n > W - v0) n = W - v0;
@@ -413,13 +430,18 @@ od_verify_stream_kernel(const VerifyArgs a)
             f += n;
             if (f >= f_hi) break;
             ++rho; v0 = 0; seg = 0;
-            if (r < mb) ++r; else find_row(a, rho, i0, i1, excl, m0, m1, b, r, mb);
+            if (r < mb) ++r; else find_row(per <= 2 ? nullptr : s_m, rho, i0, i1, excl, m0, m1, b, r, mb);
         }
     }
 
     // ---- the parked partials of space A: every warp hands over its own (its lane 0
     // wrote them), at the end, where nothing waits for it
-    if (early && a_lo < a_hi && lane == 0) {
+    if (early && lane == 0) {
+        // (the span is worked out again from the block index rather than kept in registers
+        // through the whole stream)
+        uint32_t g2 = blockIdx.x;
+        asm volatile("" : "+r"(g2));
+        span_of_space_a(a, g2, a_lo, a_hi, a_b0, a_v0, a_seg0);
         uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
         int k = 0;
         while (f < a_hi) {
