@@ -509,7 +509,8 @@ def main():
     if a.verify_grid:
         ctx.set_option("verify_grid", a.verify_grid)
     # the pool's inputs are resident long before any timed launch: od_verify called on its own
-    # (the roofline graph) may read rows 0 before it waits for the launch in front
+    # (the roofline graph) may read rows 0, and the step's translation kernel the proposal,
+    # before they wait for the launch in front
     ctx.set_option("early_inputs", 1)
     if a.sample_tiles_per_warp:
         ctx.set_option("sample_tiles_per_warp", a.sample_tiles_per_warp)
@@ -698,10 +699,13 @@ def main():
                                     f"{P * logit_bytes / 2**20:.0f} MiB of logits cycled",
                        "launch": ("K steps (one od_step call each) captured in one CUDA graph, replayed for 1.5 s; "
                                   "value from the median replay") if not a.no_graph else "eager launches",
-                       "roofline_launch": "od_verify alone, K calls in one graph, option early_inputs = 1 "
-                                          "(the pool's inputs are resident before any timed launch)",
+                       "roofline_launch": "od_verify alone, K calls in one graph",
+                       "options": "early_inputs = 1 for every launch (the pool's inputs are resident "
+                                  "before any timed launch)",
                        "parallelism": f"batch sharding x{world}, no collective"},
-            "gpu_launches": 4 * a.steps,
+            # od_step: translation, streaming pass, sampler (which takes step 2's decisions);
+            # without programmatic dependent launch the decide kernel is a launch of its own
+            "gpu_launches": (4 if a.no_pdl else 3) * a.steps,
             "kernels_ms_per_step": {"od_map_proposals": ms_k1 / a.steps, "od_verify": ms_k2 / a.steps,
                                     "od_sample_residual": ms_k3 / a.steps,
                                     "step_replays": len(extra),
