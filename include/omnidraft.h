@@ -173,7 +173,12 @@ int32_t od_cache_build(od_ctx *ctx, const int32_t *host_runs,
  * od_cache_configure installs an EMPTY online cache for at most `max_entries`
  * entries after a trim (policy 0 = LRU, 1 = LFU) and batches of at most `max_insert`
  * candidates; it replaces any earlier cache (od_cache_build does the reverse) and is
- * synchronous. Needs draft_vocab <= 65535 (UNSUPPORTED otherwise). */
+ * synchronous. Needs draft_vocab <= 65535 (UNSUPPORTED otherwise). Device memory:
+ * the table has S = the next power of two >= 2 * (max_entries + max_insert) slots;
+ * two copies of it (24 bytes per slot each, the second one is the table a trim
+ * builds), a claim word per slot and 68 bytes per slot of trim scratch are
+ * allocated here, 120 * S bytes in all (NOMEM if that fails); nothing is
+ * allocated later. */
 int32_t od_cache_configure(od_ctx *ctx, int64_t max_entries, int32_t policy,
                            int32_t max_insert);
 

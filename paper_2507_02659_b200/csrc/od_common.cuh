@@ -44,6 +44,7 @@ struct od_ctx {
     uint32_t *d_owner;              // [cap] first-wins claims of a batch (0xFFFFFFFF = none)
     int32_t *d_cand_slot;           // [dyn_max_insert]
     void *d_trim;                   // trim / size state (device)
+    void *d_trim_lists;             // trim scratch: the live entries' records and two candidate lists, 64 bytes per slot
 
     // od_verify scratch
     float4 *d_partials;             // [rows][OD_VERIFY_SEG_MAX] (c, sum, max, -), rows of one launch
