@@ -96,11 +96,35 @@ __device__ __forceinline__ unsigned int digit_of(int pass, unsigned long long hi
                     : (unsigned int)(lo >> (8 * (12 - pass))) & 0xFFu;
 }
 
+// The kernels of an insertion and of a trim form chains in which each needs what the one
+// before it wrote. They are launched with programmatic stream serialization and wait at once:
+// the launch latency of a kernel is spent while its predecessor still runs.
+__device__ __forceinline__ void chain_wait()
+{
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// launch with or without programmatic stream serialization (the context's "pdl" option)
+template <typename... Params, typename... Args>
+cudaError_t chain_launch(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t s, bool pdl, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
+
 __global__ void insert_claim_kernel(int32_t N, int32_t v_q, int32_t v_p, const int32_t *__restrict__ runs,
                                     const int32_t *__restrict__ len, const int32_t *__restrict__ target,
                                     unsigned long long *keys, const int32_t *vals, int64_t cap,
                                     unsigned int *owner, int32_t *cand_slot, TrimState *st)
 {
+    chain_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     cand_slot[i] = -1;
@@ -116,7 +140,21 @@ __global__ void insert_claim_kernel(int32_t N, int32_t v_q, int32_t v_p, const i
     const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
     uint64_t g = od_hash64(key) & (ngroups - 1);
     for (uint64_t step = 0; step < ngroups; ++step) {       // bounded: ends on any table contents
-        for (int s = 0; s < OD_GROUP; ++s) {
+        // A group is filled from slot 0 without holes, and in a table at most half full it
+        // rarely holds more than sixteen entries: its first sixteen keys are read at once
+        // (one round trip instead of one per occupied slot), the rest one by one.
+        constexpr int HEAD = 16;
+        unsigned long long head[HEAD];
+#pragma unroll
+        for (int h = 0; h < HEAD / 2; ++h) {
+            const ulonglong2 a = __ldcg((const ulonglong2 *)(keys + g * OD_GROUP) + h);
+            head[2 * h] = a.x; head[2 * h + 1] = a.y;
+        }
+        int s0 = HEAD;                                      // the first slot that is empty or holds the key
+#pragma unroll
+        for (int h = HEAD - 1; h >= 0; --h)
+            if (head[h] == 0ull || head[h] == key) s0 = h;
+        for (int s = s0; s < OD_GROUP; ++s) {
             const int64_t slot = (int64_t)(g * OD_GROUP + s);
             unsigned long long cur = keys[slot];
             if (cur == 0ull) cur = atomicCAS(keys + slot, 0ull, key);   // 0 again: the slot is ours
@@ -138,6 +176,7 @@ __global__ void insert_commit_kernel(int32_t N, const int32_t *__restrict__ targ
                                      unsigned int *owner, const int32_t *__restrict__ cand_slot,
                                      unsigned int clock, TrimState *st)
 {
+    chain_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     const int32_t slot = cand_slot[i];
@@ -147,15 +186,6 @@ __global__ void insert_commit_kernel(int32_t N, const int32_t *__restrict__ targ
     vals[slot] = target[i];                                  // the entry exists from here on
     owner[slot] = 0xFFFFFFFFu;
     atomicAdd(&st->size, 1u);
-}
-
-// The trim's kernels form a chain in which each needs what the one before it wrote. They are
-// launched with programmatic stream serialization and wait at once: the launch latency of a
-// kernel is spent while its predecessor still runs.
-__device__ __forceinline__ void chain_wait()
-{
-    asm volatile("griddepcontrol.launch_dependents;");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 __global__ void trim_begin_kernel(TrimState *st, unsigned int max_entries)
@@ -455,19 +485,6 @@ __global__ void trim_end_kernel(TrimState *st)
     st->size -= st->k; st->k = 0u;
 }
 
-// launch with or without programmatic stream serialization (the context's "pdl" option)
-template <typename... Params, typename... Args>
-cudaError_t chain_launch(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t s, bool pdl, Args... args)
-{
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
-}
-
 #define OD_CUDA(call)                                  \
     do {                                               \
         cudaError_t e__ = (call);                      \
@@ -570,12 +587,13 @@ int32_t od_cache_insert(od_ctx *c, int32_t N, const int32_t *runs, const int32_t
     cudaStream_t s = (cudaStream_t)stream;
     c->last_was_map = false;
     const int threads = 128, blocks = (N + threads - 1) / threads;
-    insert_claim_kernel<<<blocks, threads, 0, s>>>(N, c->v_q, c->v_p, runs, len, target,
-                                                   (unsigned long long *)c->d_keys, c->d_vals, c->cap,
-                                                   c->d_owner, c->d_cand_slot, (TrimState *)c->d_trim);
-    insert_commit_kernel<<<blocks, threads, 0, s>>>(N, target, c->d_vals, c->d_stamp, c->d_freq, c->d_born,
-                                                    c->d_owner, c->d_cand_slot, c->clock,
-                                                    (TrimState *)c->d_trim);
+    const bool pdl = c->opt_pdl != 0;
+    OD_CUDA(chain_launch(insert_claim_kernel, (unsigned)blocks, (unsigned)threads, s, pdl, N, c->v_q, c->v_p, runs, len,
+                         target, (unsigned long long *)c->d_keys, (const int32_t *)c->d_vals, c->cap,
+                         c->d_owner, c->d_cand_slot, (TrimState *)c->d_trim));
+    OD_CUDA(chain_launch(insert_commit_kernel, (unsigned)blocks, (unsigned)threads, s, pdl, N, target, c->d_vals,
+                         c->d_stamp, c->d_freq, c->d_born, c->d_owner, (const int32_t *)c->d_cand_slot,
+                         c->clock, (TrimState *)c->d_trim));
     OD_CUDA(cudaGetLastError());
     return OD_OK;
 }
