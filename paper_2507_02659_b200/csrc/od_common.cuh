@@ -103,7 +103,7 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
 // od_step: the streaming pass of step 2 alone (no decide kernel), and what the sampler then needs
 // to take step 2's decisions itself: the split of the pass and where step 2's outputs go.
 struct od_fused_verify {
-    int32_t W, n_chunks, span_min, span_a;
+    int32_t W, n_chunks, span_min, span_a, seg_warps;
     float *row_max, *row_sum, *p_sel, *ratio;
     int32_t *n_accepted, *n_draft_accepted;
     uint32_t *flags;

@@ -7,14 +7,13 @@
 
 #include "od_common.cuh"
 
-#define OD_STREAM_WARPS 8           // warps of a stream-kernel block: partials per block segment
-
 // The split of the streaming pass (see od_verify.cu): enough to find a row's partials.
 struct StreamPlan {
     int32_t W;                      // 512-byte units per row
     int32_t n_chunks;               // blocks of the stream grid
     int32_t span_min;               // smallest span of space B
     int32_t span_a;                 // units of space A per block
+    int32_t seg_warps;              // warps of a stream-kernel block: partials per block segment
     const float4 *partials;         // [row slot][OD_VERIFY_SEG_MAX] (c, sum, max, -)
 };
 
@@ -72,7 +71,7 @@ __device__ __forceinline__ void merge_row_partials(const StreamPlan &p, int row_
 {
     const float4 *pp = p.partials + (size_t)row_slot * OD_VERIFY_SEG_MAX;
     // at most OD_VERIFY_SEG_MAX = 64 partials: two per lane, both requested before either is used
-    const int n = nseg * OD_STREAM_WARPS;
+    const int n = nseg * p.seg_warps;
     float4 v0 = make_float4(0.f, 0.f, 0.f, 0.f), v1 = v0;
     if (lane < n) v0 = __ldcg(pp + lane);
     if (lane + 32 < n) v1 = __ldcg(pp + lane + 32);

@@ -861,7 +861,7 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     a.early = c->last_was_map ? 0 : 1;
     if (fuse) {
         a.plan.W = fuse->W; a.plan.n_chunks = fuse->n_chunks; a.plan.span_min = fuse->span_min;
-        a.plan.span_a = fuse->span_a; a.plan.partials = c->d_partials;
+        a.plan.span_a = fuse->span_a; a.plan.seg_warps = fuse->seg_warps; a.plan.partials = c->d_partials;
         a.w_row_max = fuse->row_max; a.w_row_sum = fuse->row_sum; a.w_p_sel = fuse->p_sel; a.w_ratio = fuse->ratio;
         a.w_n_accepted = fuse->n_accepted; a.w_n_draft = fuse->n_draft_accepted; a.w_vflags = fuse->flags;
     }

@@ -51,9 +51,15 @@
 
 namespace {
 
-constexpr int THREADS = 256;
-constexpr int WARPS = THREADS / 32;
-static_assert(WARPS == OD_STREAM_WARPS, "partials per block segment");
+// Two block shapes of the stream kernel. Rows of 128 KB and more (256 units) go to blocks of
+// 16 warps, two per multiprocessor: fewer blocks of different age share a multiprocessor,
+// and od_verify is 0.5 us (batched 128256-id rows) to 8 us (512 x 9 rows of 152064 ids)
+// faster; shorter rows would leave a warp of such a block less than two groups of loads per
+// row, and keep blocks of 8 warps, four per multiprocessor. The template parameter TW is
+// the number of warps; a block segment has TW partials.
+constexpr int NARROW_WARPS = 8, WIDE_WARPS = 16;
+constexpr int WIDE_MIN_UNITS = 256;
+static_assert(OD_VERIFY_SEG_MAX % WIDE_WARPS == 0 && OD_VERIFY_SEG_MAX / WIDE_WARPS >= 3, "segments per row");
 constexpr int U = 4;                            // 16-byte loads in flight per thread
 constexpr int A_PARK = 8;                       // partials of space A a block can hold back
 #ifndef OD_VERIFY_MAXNREG
@@ -69,7 +75,8 @@ struct VerifyArgs {
     int32_t B, K_max, v_p;
     int32_t W;                          // 512-byte units per row
     int32_t n_chunks;                   // blocks of the stream grid
-    int32_t span_min;                   // keeps a row within OD_VERIFY_SEG_MAX / WARPS block segments
+    int32_t seg_warps;                  // warps of a block = partials of a block segment (8 or 16)
+    int32_t span_min;                   // keeps a row within OD_VERIFY_SEG_MAX / seg_warps block segments
     int32_t span_a;                     // units of space A per block
     int32_t a_early;                    // 1: space A is streamed before griddepcontrol.wait (the caller allows
                                         // it and a block's span of space A has at most A_PARK segments)
@@ -190,11 +197,12 @@ __device__ __forceinline__ void absorb_one(Lane<DTYPE> &L, float x, float scale)
 }
 
 // the first n (1..U, the same for the whole warp) loads of a group
+template <int TW>
 __device__ __forceinline__ void load_group(uint4 (&x)[U], const uint4 *p, int n)
 {
 #pragma unroll
     for (int u = 0; u < U; ++u)
-        if (u < n) x[u] = ld_stream(p + u * WARPS * 32);
+        if (u < n) x[u] = ld_stream(p + u * TW * 32);
 }
 
 template <int DTYPE>
@@ -209,7 +217,7 @@ __device__ __forceinline__ void absorb_group(Lane<DTYPE> &L, const uint4 (&x)[U]
 
 // Units [v0, v1) of row (b, r) by the whole block; warp w stores its partial to dst[w]
 // (global or shared memory).
-template <int DTYPE>
+template <int DTYPE, int TW>
 __device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r, int v0, int v1, float4 *dst)
 {
     constexpr int VEC = DTYPE == OD_BF16 ? 8 : 4;          // elements per 16 bytes
@@ -219,7 +227,7 @@ __device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r,
     const char *row = (const char *)a.logits + ((size_t)b * a.seq_stride + (size_t)r * a.row_stride) * ESZ;
     Lane<DTYPE> L;
     L.reset();
-    // A warp owns whole units (512 bytes, 16 per lane): units v0 + warp, + WARPS, ...
+    // A warp owns whole units (512 bytes, 16 per lane): units v0 + warp, + TW, ...
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int full_vecs = a.v_p / VEC;                     // whole 16-byte vectors in the row
     const int full_units = full_vecs >> 5;                 // units whose 32 lanes are all inside
@@ -233,26 +241,26 @@ __device__ __forceinline__ void block_segment(const VerifyArgs &a, int b, int r,
     // (1..U units) and is requested like any other, one group ahead; no lane ever
     // computes on padding. Only the row's last unit can be ragged (lanes past the
     // end of the row, or a final piece under 16 bytes).
-    int cnt = v < v1f ? (v1f - v + WARPS - 1) / WARPS : 0;   // this warp's whole units
+    int cnt = v < v1f ? (v1f - v + TW - 1) / TW : 0;   // this warp's whole units
     if (cnt > 0) {
         uint4 xa[U], xb[U];
         int na = cnt < U ? cnt : U, nb = 0;
-        load_group(xa, p, na);
-        cnt -= na; p += U * WARPS * 32;
+        load_group<TW>(xa, p, na);
+        cnt -= na; p += U * TW * 32;
         for (;;) {
             if (cnt == 0) { absorb_group<DTYPE>(L, xa, na, scale); break; }
             nb = cnt < U ? cnt : U;
-            load_group(xb, p, nb);
-            cnt -= nb; p += U * WARPS * 32;
+            load_group<TW>(xb, p, nb);
+            cnt -= nb; p += U * TW * 32;
             absorb<DTYPE, U>(L, xa, scale);
             if (cnt == 0) { absorb_group<DTYPE>(L, xb, nb, scale); break; }
             na = cnt < U ? cnt : U;
-            load_group(xa, p, na);
-            cnt -= na; p += U * WARPS * 32;
+            load_group<TW>(xa, p, na);
+            cnt -= na; p += U * TW * 32;
             absorb<DTYPE, U>(L, xb, scale);
         }
     }
-    if (v1 > full_units && warp == ((full_units - v0) & (WARPS - 1))) {
+    if (v1 > full_units && warp == ((full_units - v0) & (TW - 1))) {
         // the row's ragged last unit (v1 == W here): whole vectors, then single elements
         const int i = full_units * 32 + lane;
         if (i < full_vecs) {
@@ -323,20 +331,21 @@ __device__ __forceinline__ void span_of_space_a(const VerifyArgs &a, uint32_t g,
     seg0 = g - (lo - v0) / (uint32_t)a.span_a;
 }
 
-// first of the WARPS partial slots of segment `seg` of row (b, r)
+// first of the partial slots (one per warp of a block) of segment `seg` of row (b, r)
 __device__ __forceinline__ float4 *partial_slot(const VerifyArgs &a, int b, int r, int seg)
 {
-    return a.partials + ((size_t)b * (a.K_max + 1) + r) * OD_VERIFY_SEG_MAX + seg * WARPS;
+    return a.partials + ((size_t)b * (a.K_max + 1) + r) * OD_VERIFY_SEG_MAX + seg * a.seg_warps;
 }
 
 // 56 registers, not 64: four resident blocks then leave an eighth of the SM's register
 // file free, enough for a block of the (small) kernel before or after this one in
 // the stream to be resident at the same time under programmatic dependent launch.
-template <int DTYPE>
+template <int DTYPE, int TW>
 __global__ void __maxnreg__(OD_VERIFY_MAXNREG)
 od_verify_stream_kernel(const VerifyArgs a)
 {
-    __shared__ float4 s_park[A_PARK][WARPS];
+    constexpr int THREADS = TW * 32;
+    __shared__ float4 s_park[A_PARK][TW];
     __shared__ int32_t s_m[OD_VERIFY_MAX_B];               // clamped m_b, batches of more than 64 sequences only
 
     // Flat unit indices stay below 2^31 (the launcher checks). What a block does between
@@ -364,7 +373,7 @@ od_verify_stream_kernel(const VerifyArgs a)
         while (f < a_hi) {
             uint32_t n = a_hi - f;
             if (n > W - v0) n = W - v0;
-            block_segment<DTYPE>(a, (int)b, 0, (int)v0, (int)(v0 + n), s_park[k++]);
+            block_segment<DTYPE, TW>(a, (int)b, 0, (int)v0, (int)(v0 + n), s_park[k++]);
             f += n; ++b; v0 = 0;
         }
     }
@@ -406,7 +415,7 @@ od_verify_stream_kernel(const VerifyArgs a)
         while (f < a_hi) {
             uint32_t n = a_hi - f;
             if (n > W - v0) n = W - v0;
-            block_segment<DTYPE>(a, (int)b, 0, (int)v0, (int)(v0 + n), partial_slot(a, (int)b, 0, (int)seg));
+            block_segment<DTYPE, TW>(a, (int)b, 0, (int)v0, (int)(v0 + n), partial_slot(a, (int)b, 0, (int)seg));
             f += n; ++b; v0 = 0; seg = 0;
         }
     }
@@ -426,7 +435,7 @@ od_verify_stream_kernel(const VerifyArgs a)
         for (;;) {
             uint32_t n = f_hi - f;
             if (n > W - v0) n = W - v0;
-            block_segment<DTYPE>(a, b, r, (int)v0, (int)(v0 + n), partial_slot(a, b, r, (int)seg));
+            block_segment<DTYPE, TW>(a, b, r, (int)v0, (int)(v0 + n), partial_slot(a, b, r, (int)seg));
             f += n;
             if (f >= f_hi) break;
             ++rho; v0 = 0; seg = 0;
@@ -571,6 +580,7 @@ od_verify_decide_kernel(const VerifyArgs a)
         const int row_slot = b * (a.K_max + 1) + r;
         StreamPlan plan;
         plan.partials = a.partials;
+        plan.seg_warps = a.seg_warps;
         float c, s, mx;
         merge_row_partials(plan, row_slot, nseg, lane, c, s, mx);
         if (SHARD) {
@@ -658,6 +668,15 @@ static void fast_div(uint32_t d, uint32_t &mul, uint32_t &sh)
     sh = l - 1;
 }
 
+// the stream kernel in the block shape the plan chose
+template <int DTYPE>
+static cudaError_t launch_stream(const VerifyArgs &a, cudaStream_t s, bool pdl)
+{
+    return a.seg_warps == WIDE_WARPS
+        ? launch(od_verify_stream_kernel<DTYPE, WIDE_WARPS>, (unsigned)a.n_chunks, WIDE_WARPS * 32, s, pdl, a)
+        : launch(od_verify_stream_kernel<DTYPE, NARROW_WARPS>, (unsigned)a.n_chunks, NARROW_WARPS * 32, s, pdl, a);
+}
+
 // Launch plan of the stream kernel for `nb` sequences whose rows hold `v_len` elements.
 static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_len, int32_t dtype, bool early,
                         VerifyArgs &a)
@@ -665,17 +684,20 @@ static void plan_stream(const od_ctx *c, int32_t nb, int32_t K_max, int32_t v_le
     const int64_t esz = dtype == OD_BF16 ? 2 : 4;
     const int64_t row_bytes = (int64_t)v_len * esz;
     const int32_t W = (int32_t)((row_bytes + 511) / 512);
-    // a row is cut into at most OD_VERIFY_SEG_MAX / WARPS block segments (one partial per warp each)
-    constexpr int MAX_BLOCK_SEGS = OD_VERIFY_SEG_MAX / WARPS;
+    const int32_t warps = W >= WIDE_MIN_UNITS ? WIDE_WARPS : NARROW_WARPS;
+    // a row is cut into at most OD_VERIFY_SEG_MAX / warps block segments (one partial per warp each)
+    const int MAX_BLOCK_SEGS = OD_VERIFY_SEG_MAX / warps;
     const int32_t span_min = (W + MAX_BLOCK_SEGS - 2) / (MAX_BLOCK_SEGS - 1);
     // one resident wave, and no more blocks than the most this slice can need
     const int64_t max_units = (int64_t)nb * (K_max + 1) * W;
-    int64_t grid = c->opt_verify_grid > 0 ? c->opt_verify_grid : (int64_t)c->sm_count * OD_VERIFY_BLOCKS_PER_SM;
+    // one resident wave: 32 warps per multiprocessor at 56 registers
+    int64_t grid = c->opt_verify_grid > 0 ? c->opt_verify_grid
+                                          : (int64_t)c->sm_count * OD_VERIFY_BLOCKS_PER_SM * NARROW_WARPS / warps;
     const int64_t need = max_units / span_min + 1;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
     a.B = nb; a.K_max = K_max; a.v_p = v_len;
-    a.W = W; a.n_chunks = (int32_t)grid; a.span_min = span_min;
+    a.W = W; a.n_chunks = (int32_t)grid; a.span_min = span_min; a.seg_warps = warps;
     int64_t span_a = ((int64_t)nb * W + grid - 1) / grid;
     if (span_a < span_min) span_a = span_min;
     a.span_a = (int32_t)span_a;
@@ -711,9 +733,10 @@ cudaError_t od_launch_verify_stream(od_ctx *c, int32_t B, int32_t K_max, const v
     c->info[0] = a.n_chunks;
     c->info[1] = a.span_a;
     plan->W = a.W; plan->n_chunks = a.n_chunks; plan->span_min = a.span_min; plan->span_a = a.span_a;
+    plan->seg_warps = a.seg_warps;
     const bool pdl = c->opt_pdl != 0;
-    return dtype == OD_BF16 ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)a.n_chunks, THREADS, s, pdl, a)
-                            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)a.n_chunks, THREADS, s, pdl, a);
+    return dtype == OD_BF16 ? launch_stream<OD_BF16>(a, s, pdl)
+                            : launch_stream<OD_F32>(a, s, pdl);
 }
 
 cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
@@ -747,8 +770,8 @@ cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *lo
 
         const bool pdl = c->opt_pdl != 0;
         cudaError_t e = dtype == OD_BF16
-            ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)a.n_chunks, THREADS, s, pdl, a)
-            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)a.n_chunks, THREADS, s, pdl, a);
+            ? launch_stream<OD_BF16>(a, s, pdl)
+            : launch_stream<OD_F32>(a, s, pdl);
         if (e != cudaSuccess) return e;
         const unsigned dthreads = 32u * (unsigned)(K_max + 1);
         e = dtype == OD_BF16
@@ -785,8 +808,8 @@ cudaError_t od_launch_verify_shard_stats(od_ctx *c, int32_t B, int32_t K_max, in
         c->info[1] = a.span_a;
         const bool pdl = c->opt_pdl != 0;
         cudaError_t e = dtype == OD_BF16
-            ? launch(od_verify_stream_kernel<OD_BF16>, (unsigned)a.n_chunks, THREADS, s, pdl, a)
-            : launch(od_verify_stream_kernel<OD_F32>, (unsigned)a.n_chunks, THREADS, s, pdl, a);
+            ? launch_stream<OD_BF16>(a, s, pdl)
+            : launch_stream<OD_F32>(a, s, pdl);
         if (e != cudaSuccess) return e;
         const unsigned dthreads = 32u * (unsigned)(K_max + 1);
         e = dtype == OD_BF16
