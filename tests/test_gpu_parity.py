@@ -129,6 +129,14 @@ def test_every_split_of_a_row_gives_the_same_answer(cuda_device, grid, tiles, pd
                   opts={"verify_grid": grid, "sample_tiles_per_warp": tiles, "pdl": pdl, "early_inputs": early})
 
 
+@pytest.mark.parametrize("grid,pdl,early", [(1, 1, 1), (3, 0, 0), (0, 1, 1), (101, 1, 0)])
+def test_every_split_of_a_long_row_gives_the_same_answer(cuda_device, grid, pdl, early):
+    """Rows of 128 KB and more are streamed by blocks of 16 warps (16 partials per block segment):
+    70001 bf16 ids are 274 units of 512 bytes, the last one ragged."""
+    w = _small("splitwide", v_q=3000, v_p=70001, B=4, cache_entries=500, gen_seed=0xBEEF41)
+    _run_workload(w, cuda_device, range(2), pad=True, opts={"verify_grid": grid, "pdl": pdl, "early_inputs": early})
+
+
 def test_sampler_tile_sums_on_the_batched_shape(cuda_device):
     """Pass 1 of the sampler (sums of e minus the list corrections) on 128256-id rows."""
     w = synth.scaled(synth.paper_config(4), B=48, gen_seed=0xBEEF49)
