@@ -144,3 +144,55 @@ def test_online_cache_argument_checks(cuda_device):
         big.cache_configure(10, 0, 8)                     # ids do not fit 16 bits
     assert e.value.status == -5
     big.close(); ctx.close()
+
+
+def test_translation_directly_behind_cache_writers_with_early_inputs(cuda_device):
+    """With "early_inputs" the translation kernel reads the proposal before it waits for the launch
+    in front of it, never the table. Nothing is synchronised between an insertion or a trim and
+    the translations behind it: they must see the table those leave."""
+    rng = np.random.default_rng(77)
+    v_q, v_p, B, K = 60, 300, 32, 6
+    vocab_map = np.where(rng.random(v_q) < 0.7, rng.permutation(v_p)[:v_q], -1).astype(np.int32)
+    ctx = od.Context(cuda_device, v_q, v_p, B, K)
+    ctx.set_vocab_map(vocab_map)
+    ctx.cache_configure(40, cp.LRU, 64)
+    ctx.set_option("early_inputs", 1)
+    ref = cp.DynamicCache(40, cp.LRU, v_q, v_p)
+    uruns, ulens = _universe(rng, 120, v_q)
+    utgt = rng.integers(0, v_p, size=120).astype(np.int32)
+    dev = cuda_device
+    for tick in range(1, 13):
+        ctx.cache_set_clock(tick); ref.set_clock(tick)
+        props = []
+        for _ in range(3):
+            d = rng.integers(0, v_q, size=(B, K)).astype(np.int32)
+            klen = rng.integers(0, K + 1, size=B).astype(np.int32)
+            for b in range(B):
+                e = int(rng.integers(0, 120)); L = int(ulens[e])
+                if L <= klen[b] and rng.random() < 0.9:
+                    o = int(rng.integers(0, klen[b] - L + 1)); d[b, o:o + L] = uruns[e, :L]
+            q = rng.random((B, K)).astype(np.float32)
+            props.append((d, klen, q, torch.from_numpy(d).to(dev), torch.from_numpy(klen).to(dev),
+                          torch.from_numpy(q).to(dev)))
+        pick = rng.integers(0, 120, size=30)
+        runs, lens, tg = uruns[pick].copy(), ulens[pick].copy(), utgt[pick].copy()
+        d_runs, d_lens, d_tg = (torch.from_numpy(x).to(dev) for x in (runs, lens, tg))
+        torch.cuda.synchronize()                              # every input is resident from here on
+        ctx.cache_insert(d_runs, d_lens, d_tg)
+        mp0 = od.od_map_proposals(ctx, *props[0][3:])        # directly behind the insertion
+        mp1 = od.od_map_proposals(ctx, *props[1][3:])        # behind another translation
+        ctx.cache_trim()
+        mp2 = od.od_map_proposals(ctx, *props[2][3:])        # directly behind the trim
+        torch.cuda.synchronize()
+        ref.insert_batch(runs, lens, tg)
+        for i, mp in enumerate((mp0, mp1, mp2)):
+            if i == 2:
+                ref.trim()
+            d, klen, q = props[i][:3]
+            for b in range(B):
+                tgt, qp, ss, sl, m, stop = ref.map_sequence(vocab_map, d[b, :klen[b]], q[b])
+                assert int(mp.m[b]) == m and bool(mp.tail_kind[b]) == stop, (tick, i, b)
+                assert mp.tgt_ids[b, :m].tolist() == tgt and mp.span_len[b, :m].tolist() == sl
+        _compare(ctx, ref)
+    ctx.close()
+
