@@ -46,9 +46,13 @@
  *     that the inputs of a call were complete before the launch that precedes
  *     the call was enqueued (a producer two launches back, or data resident
  *     since an earlier synchronisation): then od_verify and
- *     od_verify_shard_stats read logits and temperatures early, and
+ *     od_verify_shard_stats read logits and temperatures early;
  *     od_map_proposals and od_step read the proposal (draft ids, lengths,
- *     q_sel) early; the n-gram table is never read early. A producer that is
+ *     q_sel) early and, unless od_cache_insert or od_cache_trim was called on
+ *     the context since its last translation, probe the n-gram table early
+ *     (the table belongs to the context; the library keeps track of who writes
+ *     it); and od_step lets its streaming kernel start on logit rows 0 while the
+ *     launch in front of the step still runs. A producer that is
  *     the launch directly in front of a call (the target model's output layer,
  *     the drafter's sampling kernel) is always safe with the default
  *     "early_inputs" = 0. od_step_host copies its inputs itself and reads

@@ -270,7 +270,7 @@ int32_t od_map_proposals(od_ctx *c, int32_t B, int32_t K_max, const int32_t *dra
     DeviceGuard g(c->device);
     if (!g.ok) return OD_ERR_CUDA;
     OD_CUDA(od_launch_map(c, B, K_max, draft_ids, draft_len, q_sel, tgt_ids, q_prime, span_start,
-                          span_len, m, tail_kind, counters, c->opt_early_inputs != 0, (cudaStream_t)stream));
+                          span_len, m, tail_kind, counters, c->opt_early_inputs != 0, false, (cudaStream_t)stream));
     return OD_OK;
 }
 
@@ -346,7 +346,7 @@ int32_t od_step(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids, c
     if (!g.ok) return OD_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     OD_CUDA(od_launch_map(c, B, K_max, draft_ids, draft_len, q_sel, tgt_ids, q_prime, span_start, span_len, m,
-                          tail_kind, counters, c->opt_early_inputs != 0, s));
+                          tail_kind, counters, c->opt_early_inputs != 0, c->opt_early_inputs != 0, s));
     // The translation kernel waits for everything in front of it before it lets the next
     // kernel start, so whatever wrote the logits has finished by the time a block of the
     // stream kernel runs: rows 0 may be read before that kernel's own wait.
@@ -608,7 +608,7 @@ int32_t od_step_host(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_i
     }
     OD_CUDA(od_launch_map(c, B, K_max, c->s_draft_ids, c->s_draft_len, c->s_q_sel, c->s_tgt_ids,
                           c->s_q_prime, c->s_span_start, c->s_span_len, c->s_m, c->s_tail, nullptr,
-                          false /* the copies above are the launches in front */, s));
+                          false /* the copies above are the launches in front */, false, s));
     c->verify_early = true;     // the translation kernel is the launch in front: see od_step
     OD_CUDA(od_launch_verify(c, B, K_max, c->s_logits, logit_dtype, row_stride, seq_stride,
                              c->s_tgt_ids, c->s_q_prime, c->s_span_len, c->s_m, c->s_temperature,

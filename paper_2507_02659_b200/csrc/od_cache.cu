@@ -561,6 +561,7 @@ int32_t od_cache_configure(od_ctx *c, int64_t max_entries, int32_t policy, int32
     OD_CUDA(cudaMemset(c->d_vals2, 0xFF, (size_t)cap * sizeof(int32_t)));
     OD_CUDA(cudaMemset(c->d_owner, 0xFF, (size_t)cap * sizeof(uint32_t)));
     c->cap = cap;
+    c->table_written = true;
     c->dyn = true; c->dyn_policy = policy; c->dyn_max = max_entries; c->dyn_max_insert = max_insert;
     c->clock = 0;
     return OD_OK;
@@ -586,6 +587,7 @@ int32_t od_cache_insert(od_ctx *c, int32_t N, const int32_t *runs, const int32_t
     if (!g.ok) return OD_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     c->last_was_map = false;
+    c->table_written = true;
     const int threads = 128, blocks = (N + threads - 1) / threads;
     const bool pdl = c->opt_pdl != 0;
     OD_CUDA(chain_launch(insert_claim_kernel, (unsigned)blocks, (unsigned)threads, s, pdl, N, c->v_q, c->v_p, runs, len,
@@ -606,6 +608,7 @@ int32_t od_cache_trim(od_ctx *c, void *stream)
     if (!g.ok) return OD_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     c->last_was_map = false;
+    c->table_written = true;
     TrimState *st = (TrimState *)c->d_trim;
     const int grid = c->sm_count * 4;
     const bool pdl = c->opt_pdl != 0;

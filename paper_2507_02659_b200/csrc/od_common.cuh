@@ -63,6 +63,7 @@ struct od_ctx {
 
     // set by the entry points for the verify launch that follows: space A may be streamed early
     bool verify_early;
+    bool table_written;             // a kernel that writes the n-gram table was launched since the last translation kernel
 
     // the last launch on this context was the translation kernel, which lets the next
     // kernel start before its own outputs exist (see od_sample.cu)
@@ -88,7 +89,7 @@ struct od_ctx {
 cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids,
                           const int32_t *draft_len, const float *q_sel, int32_t *tgt_ids,
                           float *q_prime, int32_t *span_start, int32_t *span_len, int32_t *m,
-                          uint8_t *tail_kind, uint32_t *counters, bool early, cudaStream_t s);
+                          uint8_t *tail_kind, uint32_t *counters, bool early, bool release_early, cudaStream_t s);
 
 cudaError_t od_launch_verify(od_ctx *c, int32_t B, int32_t K_max, const void *logits,
                              int32_t dtype, int64_t row_stride, int64_t seq_stride,

@@ -58,80 +58,91 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // The proposal itself (ids, length, probabilities) is the caller's input. Where the
     // caller has promised that it was complete before the launch in front of this one was
-    // enqueued (early), it is requested before the wait; the table and everything this
-    // kernel writes always wait.
+    // enqueued (early bit 0), it is requested before the wait. The n-gram table and the
+    // vocabulary map belong to the context: unless a kernel that writes the table was
+    // launched on this context since the last translation kernel (early bit 1 clear), the
+    // probes run before the wait as well, and only the serial walk, which writes, is left
+    // for after it. Inside od_step (early bit 2) the next kernel is the streaming pass, which
+    // starts on logit rows 0 before its own wait (inputs under the same promise) and releases
+    // ITS successor only after that wait: it is released at once, so that rows 0 stream under
+    // the tail of the step in front.
     int K = 0;
     int32_t my_id = -1;
     float my_q = 0.f;
-    if (early && b < B) {
+    const bool early_proposal = (early & 1) != 0, early_table = (early & 2) != 0, early_release = (early & 4) != 0;
+    auto load_proposal = [&]() {
         K = draft_len[b];
         if (threadIdx.x < K_max) my_id = draft_ids[(size_t)b * K_max + threadIdx.x];
         if (lane == 0 && warp < K_max) my_q = q_sel[(size_t)b * K_max + warp];
+    };
+    auto probe = [&]() {
+        K = K < 0 ? 0 : (K > K_max ? K_max : K);
+        if (threadIdx.x < K_max) s_ids[threadIdx.x] = my_id;
+        __syncthreads();
+
+        const int s = warp;
+        if (s < K) {
+            // what the serial walk below would otherwise fetch one position at a time
+            if (lane == 0) {
+                const int32_t id = s_ids[s];
+                s_direct[s] = (id >= 0 && id < v_q) ? __ldg(vocab_map + id) : -1;
+                s_q[s] = my_q;
+            }
+            int32_t hit[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
+            int32_t slot[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
+            if (cap > 0) {
+                const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
+                uint64_t key[OD_NGRAM_MAX + 1], grp[OD_NGRAM_MAX + 1], kl[OD_NGRAM_MAX + 1];
+                int32_t vl[OD_NGRAM_MAX + 1];
+                bool valid[OD_NGRAM_MAX + 1];
+                // ids of a run must lie in the draft vocabulary; the run must fit
+                bool ok = true;
+                uint64_t k = 0;
+#pragma unroll
+                for (int L = 1; L <= OD_NGRAM_MAX; ++L) {
+                    int32_t id = (s + L - 1 < K) ? s_ids[s + L - 1] : -1;
+                    ok = ok && (s + L <= K) && id >= 0 && id < v_q;
+                    k |= (uint64_t)(uint32_t)(id + 1) << (16 * (L - 1));
+                    valid[L] = ok && L >= 2;
+                    key[L] = k;
+                    grp[L] = od_hash64(k) & (ngroups - 1);
+                }
+#pragma unroll
+                for (int L = 2; L <= OD_NGRAM_MAX; ++L) {
+                    kl[L] = valid[L] ? __ldg(keys + grp[L] * OD_GROUP + lane) : 0ULL;
+                    // the values of the group come with its keys, so a hit costs one round trip
+                    // (a concurrent batch insert writes an entry's value last: read it past L1)
+                    vl[L] = valid[L] ? __ldcg(vals + grp[L] * OD_GROUP + lane) : -1;
+                }
+#pragma unroll
+                for (int L = 2; L <= OD_NGRAM_MAX; ++L)
+                    if (valid[L]) {
+                        int32_t value = -1;
+                        slot[L] = probe_continue(keys, vals, ngroups, key[L], grp[L], kl[L], vl[L], lane, &value);
+                        // an entry whose value is not set yet does not exist
+                        if (slot[L] >= 0) hit[L] = value;
+                    }
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int L = 2; L <= OD_NGRAM_MAX; ++L) { s_hit[s][L] = hit[L]; s_slot[s][L] = slot[L]; }
+            }
+        }
+    };
+    if (early_release) asm volatile("griddepcontrol.launch_dependents;");
+    if (early_proposal && b < B) {
+        load_proposal();
+        if (early_table) probe();
     }
 
     // under programmatic dependent launch: wait for everything earlier in the
-    // stream first, only then let the verification kernel start its prefetch
+    // stream first, only then (no promise) let the verification kernel start its prefetch
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;");
+    if (!early_release) asm volatile("griddepcontrol.launch_dependents;");
 
     if (b >= B) return;
-    if (!early) {
-        K = draft_len[b];
-        if (threadIdx.x < K_max) my_id = draft_ids[(size_t)b * K_max + threadIdx.x];
-        if (lane == 0 && warp < K_max) my_q = q_sel[(size_t)b * K_max + warp];
-    }
-    K = K < 0 ? 0 : (K > K_max ? K_max : K);
-    if (threadIdx.x < K_max) s_ids[threadIdx.x] = my_id;
-    __syncthreads();
-
-    const int s = warp;
-    if (s < K) {
-        // what the serial walk below would otherwise fetch one position at a time
-        if (lane == 0) {
-            const int32_t id = s_ids[s];
-            s_direct[s] = (id >= 0 && id < v_q) ? __ldg(vocab_map + id) : -1;
-            s_q[s] = my_q;
-        }
-        int32_t hit[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
-        int32_t slot[OD_NGRAM_MAX + 1] = {-1, -1, -1, -1, -1};
-        if (cap > 0) {
-            const uint64_t ngroups = (uint64_t)cap / OD_GROUP;
-            uint64_t key[OD_NGRAM_MAX + 1], grp[OD_NGRAM_MAX + 1], kl[OD_NGRAM_MAX + 1];
-            int32_t vl[OD_NGRAM_MAX + 1];
-            bool valid[OD_NGRAM_MAX + 1];
-            // ids of a run must lie in the draft vocabulary; the run must fit
-            bool ok = true;
-            uint64_t k = 0;
-#pragma unroll
-            for (int L = 1; L <= OD_NGRAM_MAX; ++L) {
-                int32_t id = (s + L - 1 < K) ? s_ids[s + L - 1] : -1;
-                ok = ok && (s + L <= K) && id >= 0 && id < v_q;
-                k |= (uint64_t)(uint32_t)(id + 1) << (16 * (L - 1));
-                valid[L] = ok && L >= 2;
-                key[L] = k;
-                grp[L] = od_hash64(k) & (ngroups - 1);
-            }
-#pragma unroll
-            for (int L = 2; L <= OD_NGRAM_MAX; ++L) {
-                kl[L] = valid[L] ? __ldg(keys + grp[L] * OD_GROUP + lane) : 0ULL;
-                // the values of the group come with its keys, so a hit costs one round trip
-                // (a concurrent batch insert writes an entry's value last: read it past L1)
-                vl[L] = valid[L] ? __ldcg(vals + grp[L] * OD_GROUP + lane) : -1;
-            }
-#pragma unroll
-            for (int L = 2; L <= OD_NGRAM_MAX; ++L)
-                if (valid[L]) {
-                    int32_t value = -1;
-                    slot[L] = probe_continue(keys, vals, ngroups, key[L], grp[L], kl[L], vl[L], lane, &value);
-                    // an entry whose value is not set yet does not exist
-                    if (slot[L] >= 0) hit[L] = value;
-                }
-        }
-        if (lane == 0) {
-#pragma unroll
-            for (int L = 2; L <= OD_NGRAM_MAX; ++L) { s_hit[s][L] = hit[L]; s_slot[s][L] = slot[L]; }
-        }
-    }
+    if (!early_proposal) load_proposal();
+    if (!(early_proposal && early_table)) probe();
     __syncthreads();
 
     if (threadIdx.x == 0) {
@@ -186,7 +197,8 @@ od_map_kernel(int32_t B, int32_t K_max, int32_t v_q, const int32_t *__restrict__
 cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *draft_ids,
                           const int32_t *draft_len, const float *q_sel, int32_t *tgt_ids,
                           float *q_prime, int32_t *span_start, int32_t *span_len, int32_t *m,
-                          uint8_t *tail_kind, uint32_t *counters, bool early, cudaStream_t s)
+                          uint8_t *tail_kind, uint32_t *counters, bool early, bool release_early,
+                          cudaStream_t s)
 {
     if (B == 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
@@ -199,9 +211,15 @@ cudaError_t od_launch_map(od_ctx *c, int32_t B, int32_t K_max, const int32_t *dr
     cfg.attrs = attr;
     cfg.numAttrs = c->opt_pdl ? 1 : 0;
     c->last_was_map = true;
+    // A kernel that writes the table (insert, trim) may be the launch in front of this one: then
+    // the probes stay behind the wait. A translation kernel releases its successor after its
+    // wait, or (inside od_step) that successor is the streaming pass, which does: either way
+    // every later translation kernel starts after those writers are done.
+    const int32_t early_bits = early && c->opt_pdl ? (c->table_written ? 1 : 3) | (release_early ? 4 : 0) : 0;
+    c->table_written = false;
     return cudaLaunchKernelEx(&cfg, od_map_kernel, B, K_max, c->v_q, draft_ids, draft_len, q_sel,
                               (const int32_t *)c->d_vocab_map, (const uint64_t *)c->d_keys,
                               (const int32_t *)c->d_vals, c->cap, tgt_ids, q_prime, span_start,
                               span_len, m, tail_kind, counters, c->dyn ? c->d_stamp : (uint32_t *)nullptr,
-                              c->dyn ? c->d_freq : (uint32_t *)nullptr, c->clock, (int32_t)(early && c->opt_pdl));
+                              c->dyn ? c->d_freq : (uint32_t *)nullptr, c->clock, early_bits);
 }
