@@ -15,7 +15,10 @@
 //           its eight ids (with the two ids Eq. (2) singles out) and one warp sum:
 //           the tile's value. Whole tiles go in pairs, software-pipelined: the
 //           inverse-map entries of the next pair are requested before the gathers
-//           of the current pair, so a pair costs one memory round trip;
+//           of the current pair, so a pair costs one memory round trip (the
+//           entries of a warp's first pair, like everything else that does not
+//           depend on the verification kernels, are requested before the kernel
+//           waits for them);
 //   ticket  blocks never wait for each other: the block that draws the
 //           sequence's last ticket continues alone;
 //   pass 2  that block scans the tile values in parallel (total,

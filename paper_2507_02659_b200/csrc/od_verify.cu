@@ -5,8 +5,9 @@
 // Two launches.
 //
 // (1) od_verify_stream_kernel: one streaming pass in which every logit crosses
-// HBM exactly once (128-bit loads, four in flight per thread, four 256-thread
-// blocks per SM: one resident wave). The bytes are split evenly over the
+// HBM exactly once (128-bit loads, four in flight per thread, one resident wave of
+// 32 warps per SM: two blocks of 16 warps for rows of 128 KB and more, four blocks
+// of 8 warps for shorter rows). The bytes are split evenly over the
 // blocks, whatever the mix of row counts. The unit of work is 512 contiguous
 // bytes of a row; a row has W units; the rows to read are laid end to end in
 // two flat index spaces and every block takes one contiguous span of each:
@@ -16,12 +17,12 @@
 //            span before it waits for the launch in front (programmatic
 //            dependent launch): the translation kernel, or the previous
 //            launch's decide kernel, is hidden behind useful traffic;
-//   space B  rows 1..m_b, split by the prefix sums of m, which every block
-//            rebuilds in shared memory (at most 2048 sequences per launch).
+//   space B  rows 1..m_b, split by the prefix sums of m, which every warp
+//            works out for itself (at most 2048 sequences per launch).
 // A span is cut at row ends into segments; every warp of the block reduces its
 // share of a segment to one partial (reference exponent c, sum of
 // exp2(x*scale - c), exact maximum) and stores it. No atomics, no fences, no
-// barriers: no warp waits for another.
+// barriers in the stream: no warp waits for another.
 //
 // (2) od_verify_decide_kernel: one block per sequence, one warp per row. Before
 // it waits for the stream kernel it loads what does not depend on it (m, T,
