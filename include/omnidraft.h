@@ -52,7 +52,11 @@
  *     the context since its last translation, probe the n-gram table early
  *     (the table belongs to the context; the library keeps track of who writes
  *     it); and od_step lets its streaming kernel start on logit rows 0 while the
- *     launch in front of the step still runs. A producer that is
+ *     launch in front of the step still runs. What the library keeps track of
+ *     it knows at the time of the call: a CUDA graph that captured
+ *     od_map_proposals or od_step under "early_inputs" = 1 must not be launched
+ *     directly behind od_cache_insert or od_cache_trim (any launch in between
+ *     that is not programmatic, or an event, restores the order). A producer that is
  *     the launch directly in front of a call (the target model's output layer,
  *     the drafter's sampling kernel) is always safe with the default
  *     "early_inputs" = 0. od_step_host copies its inputs itself and reads
