@@ -390,9 +390,26 @@ od_verify_stream_kernel(const VerifyArgs a)
 
     // ---- rows of space B before each lane's sequences, and in all
     uint32_t loc = 0, m0 = 0, m1 = 0;
+    int32_t raw0 = 0, raw1 = 0;
     if (per <= 2) {
-        if (i0 < i1) m0 = (uint32_t)clamp_m(a.m[i0], a.K_max);
-        if (i0 + 1 < i1) m1 = (uint32_t)clamp_m(a.m[i0 + 1], a.K_max);
+        if (i0 < i1) raw0 = a.m[i0];
+        if (i0 + 1 < i1) raw1 = a.m[i0 + 1];
+    }
+    // ---- the parked partials of space A: every warp hands over its own (its lane 0 wrote
+    // them) while the loads of m are on their way: the warp has nothing else to do
+    if (early && lane == 0) {
+        uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
+        int k = 0;
+        while (f < a_hi) {
+            uint32_t n = a_hi - f;
+            if (n > W - v0) n = W - v0;
+            partial_slot(a, (int)b, 0, (int)seg)[warp] = s_park[k][warp];
+            ++k; f += n; ++b; v0 = 0; seg = 0;
+        }
+    }
+    if (per <= 2) {
+        m0 = (uint32_t)clamp_m(raw0, a.K_max);
+        m1 = (uint32_t)clamp_m(raw1, a.K_max);
         loc = m0 + m1;
     } else {
         // more than 64 sequences: the block reads m once into shared memory (a load that is
@@ -441,24 +458,6 @@ od_verify_stream_kernel(const VerifyArgs a)
             if (f >= f_hi) break;
             ++rho; v0 = 0; seg = 0;
             if (r < mb) ++r; else find_row(per <= 2 ? nullptr : s_m, rho, i0, i1, excl, m0, m1, b, r, mb);
-        }
-    }
-
-    // ---- the parked partials of space A: every warp hands over its own (its lane 0
-    // wrote them), at the end, where nothing waits for it
-    if (early && lane == 0) {
-        // (the span is worked out again from the block index rather than kept in registers
-        // through the whole stream)
-        uint32_t g2 = blockIdx.x;
-        asm volatile("" : "+r"(g2));
-        span_of_space_a(a, g2, a_lo, a_hi, a_b0, a_v0, a_seg0);
-        uint32_t f = a_lo, b = a_b0, v0 = a_v0, seg = a_seg0;
-        int k = 0;
-        while (f < a_hi) {
-            uint32_t n = a_hi - f;
-            if (n > W - v0) n = W - v0;
-            partial_slot(a, (int)b, 0, (int)seg)[warp] = s_park[k][warp];
-            ++k; f += n; ++b; v0 = 0; seg = 0;
         }
     }
 }
