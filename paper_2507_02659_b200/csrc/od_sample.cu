@@ -366,6 +366,7 @@ od_sample_kernel(const SampleArgs a)
     __shared__ unsigned int s_last;
     __shared__ int s_tile, s_lastmass, s_token;
     __shared__ double s_before, s_total;
+    __shared__ double s_cross[OD_SAMPLE_THREADS];           // pass 2: the sum in front of a thread's crossing tile
 
     const int b = blockIdx.y;
     const int K = a.K_max;
@@ -699,11 +700,15 @@ od_sample_kernel(const SampleArgs a)
         if (lane == 31) s_warp[warp] = inc;
         if (threadIdx.x == 0) { s_tile = 0x7FFFFFFF; s_lastmass = -1; s_token = -2; }
         __syncthreads();
-        double base = MODE == 2 ? shard_before : 0.0;
-        for (int w = 0; w < warp; ++w) base += s_warp[w];
-        if (threadIdx.x == OD_SAMPLE_THREADS - 1) s_total = base + inc;
-        __syncthreads();
-        const double Rn = MODE == 2 ? shard_total : s_total;   // unnormalised total
+        // every thread adds the warps' sums up itself (the same order everywhere): no barrier
+        // for the total
+        double base = MODE == 2 ? shard_before : 0.0, tot = 0.0;
+        for (int w = 0; w < WARPS; ++w) {
+            if (w == warp) base += tot;
+            tot += s_warp[w];
+        }
+        if (threadIdx.x == 0) s_total = tot;
+        const double Rn = MODE == 2 ? shard_total : tot;   // unnormalised total
         double target = 0.0;
         if (Rn > 0.0) {
             target = (double)u * Rn;
@@ -712,7 +717,13 @@ od_sample_kernel(const SampleArgs a)
             for (int t = my_lo; t < my_hi; ++t) {
                 const double v = s_val[t];
                 if (v > 0.0) last = t;
-                if (c + v > target) { atomicMin(&s_tile, t); break; }   // first crossing of this run
+                if (c + v > target) {
+                    // first crossing of this run: the tile, and with it who found it, so that
+                    // the sum before the tile needs no barrier of its own
+                    s_cross[threadIdx.x] = c;
+                    atomicMin(&s_tile, t * OD_SAMPLE_THREADS + (int)threadIdx.x);
+                    break;
+                }
                 c += v;
             }
             if (last >= 0) atomicMax(&s_lastmass, last);
@@ -720,13 +731,22 @@ od_sample_kernel(const SampleArgs a)
         __syncthreads();
         // cumulative sums never decrease, so the smallest reported tile is the crossing;
         // if rounding hid it, take the last tile that has mass
-        const int t_pick = Rn > 0.0 ? (s_tile != 0x7FFFFFFF ? s_tile : s_lastmass) : -1;
-        if (t_pick >= my_lo && t_pick < my_hi) {    // its owner publishes the sum before it
-            double c = base + inc - loc;
-            for (int t = my_lo; t < t_pick; ++t) c += s_val[t];
-            s_before = c;
+        int t_pick = -1;
+        if (Rn > 0.0) {
+            if (s_tile != 0x7FFFFFFF) {
+                t_pick = s_tile / OD_SAMPLE_THREADS;
+                if (threadIdx.x < 32) s_before = s_cross[s_tile % OD_SAMPLE_THREADS];   // warp 0 reads it back below
+                __syncwarp();
+            } else {
+                t_pick = s_lastmass;
+                if (t_pick >= my_lo && t_pick < my_hi) {    // its owner publishes the sum before it
+                    double c = base + inc - loc;
+                    for (int t = my_lo; t < t_pick; ++t) c += s_val[t];
+                    s_before = c;
+                }
+                __syncthreads();                            // (block-uniform: s_tile is the same for all)
+            }
         }
-        __syncthreads();
         if (t_pick >= 0 && warp == 0) {
             // ---- warp 0 evaluates the chosen tile id by id and scans inside it ----
             float r[EPT];
