@@ -204,7 +204,7 @@ int32_t od_cache_set_clock(od_ctx *ctx, uint32_t clock);
  * The table is sized for max_entries + max_insert entries at load 1/2: trim at
  * least once per batch that can take the cache past max_entries. A candidate that
  * finds no free slot on its whole probe sequence (only possible when trims were
- * skipped for many batches) is dropped without a trace. */
+ * skipped for many batches) is dropped and counted (od_cache_stats). */
 int32_t od_cache_insert(od_ctx *ctx, int32_t N, const int32_t *runs,
                         const int32_t *len, const int32_t *target, void *stream);
 
@@ -218,6 +218,14 @@ int32_t od_cache_insert(od_ctx *ctx, int32_t N, const int32_t *runs,
  * clock of its capture and must be captured again after od_cache_trim or
  * od_cache_set_clock. */
 int32_t od_cache_trim(od_ctx *ctx, void *stream);
+
+/* Counters of the online cache since od_cache_configure (synchronises the device; any
+ * pointer may be NULL): the number of entries; the malformed candidates od_cache_insert
+ * skipped; the candidates it lost because their whole probe sequence was full, which
+ * happens only when trims were skipped for so long that the table filled up (Algorithm 1's
+ * cache update has no such case: the paper's cache is unbounded unless trimmed, App. D.5).
+ * STATE without an online cache. */
+int32_t od_cache_stats(od_ctx *ctx, int64_t *entries, int64_t *invalid, int64_t *dropped);
 
 /* Contents of the online cache, for inspection and tests: synchronises the device,
  * writes up to max_out entries (host arrays: runs int32[max_out,4] padded with -1,

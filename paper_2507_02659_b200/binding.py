@@ -32,7 +32,7 @@ OD_NOALLOC_MAX_ROWS = 1024
 EXPORTS = ["od_create", "od_destroy", "od_set_vocab_map", "od_cache_build", "od_set_option",
            "od_map_proposals", "od_verify", "od_sample_residual", "od_step", "od_host_step_reserve",
            "od_step_host", "od_verify_noalloc", "od_exit_rule", "od_cache_configure", "od_cache_set_clock",
-           "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_distill_loss",
+           "od_cache_insert", "od_cache_trim", "od_cache_dump", "od_cache_stats", "od_distill_loss",
            "od_verify_shard_stats", "od_verify_shard_finish", "od_sample_shard_mass", "od_sample_shard_pick",
            "od_last_launch_info", "od_status_string", "od_version"]
 
@@ -81,6 +81,7 @@ def lib():
         L.od_cache_insert.argtypes = [vp, i32, vp, vp, vp, vp]
         L.od_cache_trim.argtypes = [vp, vp]
         L.od_cache_dump.argtypes = [vp, i64, vp, vp, vp, vp, vp, C.POINTER(i64)]
+        L.od_cache_stats.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
         L.od_host_step_reserve.argtypes = [vp, i32]
         L.od_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, vp, u64] + [vp] * 7 + [vp]
         L.od_last_launch_info.argtypes = [vp, i32]
@@ -188,6 +189,12 @@ class Context:
 
     def cache_trim(self):
         _check(lib().od_cache_trim(self.handle, _stream(self.device)), "od_cache_trim")
+
+    def cache_stats(self):
+        """(entries, malformed candidates skipped, candidates lost to a full table) of the online cache."""
+        e, i, d = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+        _check(lib().od_cache_stats(self.handle, C.byref(e), C.byref(i), C.byref(d)), "od_cache_stats")
+        return e.value, i.value, d.value
 
     def cache_dump(self):
         """{run tuple: (target, last-access clock, frequency)} of the online cache (synchronous)."""

@@ -27,6 +27,7 @@
 //           digit of (new?, score) that is the same in every live entry costs no
 //           histogram at all. Then the survivors are re-inserted from the dense list
 //           into the spare table, which becomes the table. No kernel waits for another.
+#include <stddef.h>
 #include <string.h>
 #include <utility>
 #include <vector>
@@ -51,6 +52,7 @@ struct TrimState {
     unsigned int size;          // live entries of the current table
     unsigned int k;             // entries to drop in this trim
     unsigned int invalid;       // malformed candidates seen by od_cache_insert
+    unsigned int dropped;       // candidates that found no free slot on their whole probe sequence
     unsigned int n_live;        // entries of the dense list
     unsigned long long hi_and, hi_or;   // AND / OR of (new?, score) over the live entries: bits that never vary
     SelState sel[PASSES + 1];   // sel[p]: written by block 0 of pass p (sel[PASSES]: by the rebuild)
@@ -169,6 +171,7 @@ __global__ void insert_claim_kernel(int32_t N, int32_t v_q, int32_t v_p, const i
         }
         g = (g + 1) & (ngroups - 1);
     }
+    atomicAdd(&st->dropped, 1u);                            // the table is full: the candidate is lost
 }
 
 __global__ void insert_commit_kernel(int32_t N, const int32_t *__restrict__ target, int32_t *vals,
@@ -628,6 +631,24 @@ int32_t od_cache_trim(od_ctx *c, void *stream)
     // the rebuilt table is the table for every call enqueued from now on
     std::swap(c->d_keys, c->d_keys2); std::swap(c->d_vals, c->d_vals2);
     std::swap(c->d_stamp, c->d_stamp2); std::swap(c->d_freq, c->d_freq2); std::swap(c->d_born, c->d_born2);
+    return OD_OK;
+}
+
+int32_t od_cache_stats(od_ctx *c, int64_t *entries, int64_t *invalid, int64_t *dropped)
+{
+    if (!c) return OD_ERR_INVALID_ARG;
+    if (!c->dyn) return OD_ERR_STATE;
+    Guard g(c->device);
+    if (!g.ok) return OD_ERR_CUDA;
+    OD_CUDA(cudaDeviceSynchronize());
+    unsigned int size = 0, inv = 0, drop = 0;
+    const char *st = (const char *)c->d_trim;
+    OD_CUDA(cudaMemcpy(&size, st + offsetof(TrimState, size), sizeof(size), cudaMemcpyDeviceToHost));
+    OD_CUDA(cudaMemcpy(&inv, st + offsetof(TrimState, invalid), sizeof(inv), cudaMemcpyDeviceToHost));
+    OD_CUDA(cudaMemcpy(&drop, st + offsetof(TrimState, dropped), sizeof(drop), cudaMemcpyDeviceToHost));
+    if (entries) *entries = size;
+    if (invalid) *invalid = inv;
+    if (dropped) *dropped = drop;
     return OD_OK;
 }
 

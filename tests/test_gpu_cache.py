@@ -196,3 +196,36 @@ def test_translation_directly_behind_cache_writers_with_early_inputs(cuda_device
         _compare(ctx, ref)
     ctx.close()
 
+
+def test_a_full_table_counts_what_it_loses(cuda_device):
+    """Insertions without a trim until the table (64 slots for a bound of 8 + 8) is full: every
+    candidate is either in the cache or counted as lost, and malformed ones are counted too."""
+    rng = np.random.default_rng(5)
+    v_q, v_p = 200, 300
+    ctx = od.Context(cuda_device, v_q, v_p, 4, 4)
+    ctx.set_vocab_map(np.full(v_q, -1, np.int32))
+    ctx.cache_configure(8, cp.LRU, 8)
+    seen = set()
+    bad = 0
+    for tick in range(1, 16):
+        ctx.cache_set_clock(tick)
+        runs = np.full((8, 4), -1, np.int32); lens = np.full(8, 2, np.int32)
+        for i in range(8):
+            while True:
+                r = tuple(int(x) for x in rng.integers(0, v_q, size=2))
+                if r not in seen:
+                    break
+            seen.add(r); runs[i, :2] = r
+        tg = rng.integers(0, v_p, size=8).astype(np.int32)
+        if tick == 3:
+            lens[0] = 7; seen.discard(tuple(int(x) for x in runs[0, :2])); bad += 1
+        ctx.cache_insert(torch.from_numpy(runs).to(cuda_device), torch.from_numpy(lens).to(cuda_device),
+                         torch.from_numpy(tg).to(cuda_device))
+    entries, invalid, dropped = ctx.cache_stats()
+    held = ctx.cache_dump()
+    assert invalid == bad
+    assert entries == len(held) == 64                 # every slot taken
+    assert dropped == len(seen) - 64 and dropped > 0
+    assert set(held) <= seen
+    ctx.close()
+
