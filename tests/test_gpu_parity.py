@@ -288,6 +288,52 @@ def test_a_producer_directly_in_front_of_the_step_is_safe(cuda_device):
     ctx.close()
 
 
+def test_a_producer_that_releases_its_dependents_before_it_writes(cuda_device):
+    """The launch directly in front of the library's first kernel is a kernel that executes
+    griddepcontrol.launch_dependents first and writes the logits (over NaN) half a millisecond
+    later, as an output-layer GEMM built for programmatic dependent launch does, only slower: the
+    library's kernels are resident and past their prologues long before the logits exist.
+    With the default options every library kernel that reads the logits must still see them:
+    od_step, od_verify on its own and od_verify_noalloc against the oracle, every time."""
+    import helpers
+    prod = helpers.early_producer_lib()
+    w = _small("earlyproducer", B=48, v_q=3000, v_p=40000, cache_entries=1000, gen_seed=0xBEEF68)
+    st = synth.make_static(w)
+    ctx = parity.make_context(w, st, cuda_device)
+    cache = oracle.Cache(st.runs, st.run_len, st.run_target)
+    s = synth.make_step(w, st, 0, device=cuda_device)
+    clean = s.logits.clone()
+    nbytes = clean.numel() * clean.element_size()
+    assert nbytes % 16 == 0
+    stream = torch.cuda.current_stream(cuda_device).cuda_stream
+    ref = None
+    for rep in range(18):
+        which = rep % 3
+        mp = od.alloc_map_out(ctx, w.B, w.k_max)
+        if which != 0:
+            od.od_map_proposals(ctx, s.draft_ids, s.draft_len, s.q_sel, out=mp)
+        vo = od.alloc_verify_out(ctx, w.B, w.k_max)
+        so = od.alloc_sample_out(ctx, w.B)
+        s.logits.fill_(float("nan"))
+        torch.cuda.synchronize()
+        assert prod.early_producer(s.logits.data_ptr(), clean.data_ptr(), nbytes, 1000000, stream) == 0
+        if which == 0:
+            od.od_step(ctx, s.draft_ids, s.draft_len, s.q_sel, s.q_rows, s.logits, s.temperature, s.seed, s.step,
+                       mp=mp, vo=vo, so=so)
+        else:
+            if which == 1:
+                od.od_verify(ctx, s.logits, mp, s.temperature, s.seed, s.step, out=vo)
+            else:
+                od.od_verify_noalloc(w.v_p, s.logits, mp, s.temperature, s.seed, s.step, out=vo)
+            od.od_sample_residual(ctx, s.logits, vo, s.q_rows, s.draft_ids, mp, s.temperature, s.seed, s.step, out=so)
+        torch.cuda.synchronize()
+        if ref is None:
+            ref = parity.oracle_step(cache, st, w, s.to("cpu"), probe=so.out_token.cpu().numpy())
+        parity.compare(mp, vo, so, ref, s.draft_len.cpu().numpy(), s.step,
+                       s.seed.cpu().numpy().astype(np.uint64), bf16=True)
+    ctx.close()
+
+
 def test_od_step_equals_the_three_calls(cuda_device):
     w = _small("onecall", B=40, v_q=3000, v_p=30011, cache_entries=800, gen_seed=0xBEEF67)
     st = synth.make_static(w)
