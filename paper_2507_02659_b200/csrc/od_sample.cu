@@ -51,6 +51,17 @@ namespace {
 constexpr int WARPS = OD_SAMPLE_THREADS / 32;
 constexpr int EPT = OD_SAMPLE_TILE / 32;                  // ids per lane per tile (8)
 
+// A 16-byte load of logits, which are read once: past L1, whose lines are better spent on the
+// drafter's row, which the gathers come back to, and on the inverse map, which the blocks of
+// other sequences on the same multiprocessor read too (od_sample_residual 14.7 -> 14.2 us on
+// the batched workload; the inverse map past L1 as well: 15.5 us).
+__device__ __forceinline__ uint4 ld_once(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
 struct SampleArgs {
     const void *logits;
     int64_t row_stride, seq_stride;
@@ -137,7 +148,7 @@ __device__ __forceinline__ void tile_values(const SeqState &q, const SampleArgs 
     if (t0 + EPT <= a.v_p) {
         float x[EPT];
         if (DTYPE == OD_BF16) {
-            const uint4 v = __ldg((const uint4 *)(q.row + (size_t)t0 * 2));
+            const uint4 v = ld_once(q.row + (size_t)t0 * 2);
             x[0] = od_bf16_lo(v.x); x[1] = od_bf16_hi(v.x); x[2] = od_bf16_lo(v.y); x[3] = od_bf16_hi(v.y);
             x[4] = od_bf16_lo(v.z); x[5] = od_bf16_hi(v.z); x[6] = od_bf16_lo(v.w); x[7] = od_bf16_hi(v.w);
         } else {
@@ -196,7 +207,7 @@ __device__ __forceinline__ void tile_e_values(const SeqState &q, const SampleArg
     if (t0 + EPT <= a.v_p) {
         float x[EPT];
         if (DTYPE == OD_BF16) {
-            const uint4 v = __ldg((const uint4 *)(q.row + (size_t)t0 * 2));
+            const uint4 v = ld_once(q.row + (size_t)t0 * 2);
             x[0] = od_bf16_lo(v.x); x[1] = od_bf16_hi(v.x); x[2] = od_bf16_lo(v.y); x[3] = od_bf16_hi(v.y);
             x[4] = od_bf16_lo(v.z); x[5] = od_bf16_hi(v.z); x[6] = od_bf16_lo(v.w); x[7] = od_bf16_hi(v.w);
         } else {
@@ -295,8 +306,8 @@ __device__ __forceinline__ void warp_tiles_dense_piped(const SeqState &q, const 
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const uint4 *src = (const uint4 *)(q.row + (size_t)((i == 0 || two ? t + i : t) * OD_SAMPLE_TILE + lane * EPT) * ESZ);
-            raw[i][0] = __ldg(src);
-            if (DTYPE != OD_BF16) raw[i][1] = __ldg(src + 1);
+            raw[i][0] = ld_once(src);
+            if (DTYPE != OD_BF16) raw[i][1] = ld_once(src + 1);
         }
         float qq[2][EPT];
 #pragma unroll
