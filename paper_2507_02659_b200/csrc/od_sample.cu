@@ -379,7 +379,11 @@ od_sample_kernel(const SampleArgs a)
     __shared__ double s_before, s_total;
     __shared__ double s_cross[OD_SAMPLE_THREADS];           // pass 2: the sum in front of a thread's crossing tile
 
-    const int b = blockIdx.y;
+    // grid = (sequences, parts of a row): blocks with neighbouring indices, which often end up on
+    // one multiprocessor, then work on the same tiles of different sequences and share the
+    // inverse-map entries in L1
+    const int b = blockIdx.x;
+    const unsigned int part = blockIdx.y, nparts = gridDim.y;
     const int K = a.K_max;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
@@ -465,7 +469,7 @@ od_sample_kernel(const SampleArgs a)
     const int tile_lo = MODE == 0 ? 0 : a.tile_lo;
     const int tile_hi = MODE == 0 ? a.ntiles : a.tile_hi;
     // pass 1's whole tiles of this warp, and the inverse-map entries of their first pair
-    const int p_lo = tile_lo + (blockIdx.x * WARPS + warp) * a.tiles_per_warp;
+    const int p_lo = tile_lo + ((int)part * WARPS + warp) * a.tiles_per_warp;
     int p_hi = p_lo + a.tiles_per_warp;
     if (p_hi > tile_hi) p_hi = tile_hi;
     const int p_hi_w = p_hi < a.v_p / OD_SAMPLE_TILE ? p_hi : a.v_p / OD_SAMPLE_TILE;
@@ -487,7 +491,7 @@ od_sample_kernel(const SampleArgs a)
             if (lane == 0) {
                 const float S = row_sum_of(c, sum, mx, dscale);
                 s_M[r] = mx; s_S[r] = S;
-                if (blockIdx.x == 0) { a.w_row_max[row_slot] = mx; a.w_row_sum[row_slot] = S; }
+                if (part == 0) { a.w_row_max[row_slot] = mx; a.w_row_sum[row_slot] = S; }
                 if (!(S > 0.f) || !(S <= FLT_MAX)) atomicOr(&s_vbits, 1u);
             }
         }
@@ -505,7 +509,7 @@ od_sample_kernel(const SampleArgs a)
             const unsigned int accmask = __ballot_sync(0xFFFFFFFFu, acc);
             while (n < mb && (accmask >> n & 1u)) ++n;
             if (bad_T) n = 0;
-            if (blockIdx.x == 0 && warp == 0) {
+            if (part == 0 && warp == 0) {
                 if (lane < mb) { a.w_p_sel[(size_t)b * K + lane] = d.p; a.w_ratio[(size_t)b * K + lane] = d.ratio; }
                 const unsigned int bndmask = __ballot_sync(0xFFFFFFFFu, bnd);
                 int nd = lane < n ? d_span : 0;
@@ -523,7 +527,7 @@ od_sample_kernel(const SampleArgs a)
     }
 
     if (!(T > 0.f)) {                              // every block of the sequence leaves here
-        if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (part == 0 && threadIdx.x == 0) {
             if (MODE == 1) {
                 a.mass_out[2 * b] = 0.0; a.mass_out[2 * b + 1] = 0.0;
             } else {
@@ -569,8 +573,8 @@ od_sample_kernel(const SampleArgs a)
             // this block's share of the drafter's row into L2 meanwhile
             if (MODE != 2 && threadIdx.x == 0) {
                 const size_t row_bytes = (size_t)a.v_q * 4 / 16 * 16;
-                size_t lo = (row_bytes / gridDim.x * blockIdx.x) / 16 * 16;
-                size_t hi = blockIdx.x + 1 == gridDim.x ? row_bytes : (row_bytes / gridDim.x * (blockIdx.x + 1)) / 16 * 16;
+                size_t lo = (row_bytes / nparts * part) / 16 * 16;
+                size_t hi = part + 1 == nparts ? row_bytes : (row_bytes / nparts * (part + 1)) / 16 * 16;
                 const char *base = (const char *)q.q_row;
                 if (((uintptr_t)base & 15u) == 0 && hi > lo)
                     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + lo), "r"((uint32_t)(hi - lo)) : "memory");
@@ -611,7 +615,7 @@ od_sample_kernel(const SampleArgs a)
         __syncthreads();
         if (threadIdx.x == 0) {
             __threadfence();
-            s_last = atomicAdd(a.ticket + b, 1u) == gridDim.x - 1 ? 1u : 0u;
+            s_last = atomicAdd(a.ticket + b, 1u) == nparts - 1 ? 1u : 0u;
             __threadfence();
         }
         __syncthreads();
@@ -906,7 +910,7 @@ static cudaError_t launch_sample(od_ctx *c, int mode, int32_t B, int32_t K_max, 
     }
 
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)blocks_x, (unsigned)B);
+    cfg.gridDim = dim3((unsigned)B, (unsigned)blocks_x);
     cfg.blockDim = dim3(OD_SAMPLE_THREADS);
     cfg.dynamicSmemBytes = od_sample_smem_bytes(ntiles);
     cfg.stream = s;
